@@ -1,0 +1,387 @@
+// Plan construction and the C ABI of the transform calls (see include/cqt.h).
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <map>
+#include <new>
+
+#include "../../include/cqt.h"
+#include "internal.hpp"
+
+using namespace cqt;
+
+namespace {
+
+const double kPi = 3.14159265358979323846;
+
+uint32_t magic_of(uint32_t d) { return d <= 1 ? 0u : (uint32_t)(((1ull << 32) + d - 1) / d); }
+
+// two-level table of exp(-2 pi i y / n), 0 <= y < n, appended to tw; returns offset and log2 C
+int append_twiddles(std::vector<float2> &tw, int64_t n, int &logC) {
+    logC = 0;
+    while ((1ll << (2 * logC)) < n) ++logC;
+    const int64_t C = 1ll << logC;
+    const int64_t nhi = (n + C - 1) / C;
+    const int off = (int)tw.size();
+    for (int64_t j = 0; j < C; ++j) {
+        const double ang = -2.0 * kPi * (double)(j % n) / (double)n;
+        tw.push_back(make_float2((float)std::cos(ang), (float)std::sin(ang)));
+    }
+    for (int64_t i = 0; i < nhi; ++i) {
+        const double ang = -2.0 * kPi * (double)((i * C) % n) / (double)n;
+        tw.push_back(make_float2((float)std::cos(ang), (float)std::sin(ang)));
+    }
+    return off;
+}
+
+const int kBandRadices[] = {16, 15, 12, 10, 9, 8, 6, 5, 4, 3, 2};
+const int kPow2Radices[] = {32, 16, 8, 4, 2};
+
+// fewest stages, then smallest largest radix
+bool best_split(int64_t m, const int *radices, int nr, std::map<int64_t, std::vector<int>> &memo, std::vector<int> &out) {
+    if (m == 1) { out.clear(); return true; }
+    auto it = memo.find(m);
+    if (it != memo.end()) { out = it->second; return !out.empty(); }
+    std::vector<int> best;
+    for (int i = 0; i < nr; ++i) {
+        const int r = radices[i];
+        if (m % r) continue;
+        std::vector<int> sub;
+        if (!best_split(m / r, radices, nr, memo, sub)) continue;
+        sub.push_back(r);
+        std::sort(sub.begin(), sub.end(), [](int a, int b) { return a > b; });
+        if (best.empty() || sub.size() < best.size() || (sub.size() == best.size() && sub[0] < best[0])) best = sub;
+    }
+    memo[m] = best;
+    out = best;
+    return !best.empty();
+}
+
+// returns false if M cannot be planned
+bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp) {
+    std::memset(&fp, 0, sizeof(fp));
+    fp.M = (int32_t)M;
+    int64_t smooth = M, rest = 1;
+    if (!pow2) {
+        smooth = 1;
+        int64_t m = M;
+        for (int p : {2, 3, 5})
+            while (m % p == 0) { m /= p; smooth *= p; }
+        rest = m;
+        if (rest > 4096) return false;
+    }
+    std::map<int64_t, std::vector<int>> memo;
+    std::vector<int> radices;
+    if (!best_split(smooth, pow2 ? kPow2Radices : kBandRadices, pow2 ? 5 : 11, memo, radices)) return false;
+    if (rest > 1) { radices.insert(radices.begin(), (int)rest); fp.generic = 1; }
+    if (radices.empty()) radices.push_back(1);
+    if ((int)radices.size() > kMaxStages) return false;
+    fp.nstages = (int32_t)radices.size();
+    int64_t n_cur = M;
+    for (int j = 0; j < fp.nstages; ++j) {
+        fp.radix[j] = radices[j];
+        fp.stride[j] = (int32_t)(n_cur / radices[j]);
+        fp.rmagic[j] = magic_of((uint32_t)radices[j]);
+        fp.smagic[j] = magic_of((uint32_t)fp.stride[j]);
+        n_cur /= radices[j];
+    }
+    int logC;
+    fp.tw_off = append_twiddles(tw, M, logC);
+    fp.logC = logC;
+    return true;
+}
+
+template <class T>
+cudaError_t upload(T *&dst, const std::vector<T> &src) {
+    dst = nullptr;
+    if (src.empty()) return cudaSuccess;
+    cudaError_t e = cudaMalloc((void **)&dst, src.size() * sizeof(T));
+    if (e != cudaSuccess) return e;
+    return cudaMemcpy(dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+void free_device(cqt_plan *p) {
+    if (p->device < 0) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    cudaSetDevice(p->device);
+    cudaFree(p->d.bands); cudaFree(p->d.ffts); cudaFree(p->d.tw);
+    cudaFree(p->d.tab_analysis); cudaFree(p->d.tab_synthesis);
+    cudaFree(p->d.tab_analysis_adj); cudaFree(p->d.tab_synthesis_adj);
+    cudaFree(p->d.cover); cudaFree(p->d.span);
+    for (auto &c : p->cls) cudaFree(c.d_work);
+    cudaSetDevice(cur);
+}
+
+bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char *cqt_status_string(cqt_status s) {
+    switch (s) {
+        case CQT_OK: return "ok";
+        case CQT_ERR_INVALID_ARG: return "invalid argument";
+        case CQT_ERR_UNSUPPORTED: return "unsupported size or layout";
+        case CQT_ERR_BAD_LAYOUT: return "band layout is not a painless frame";
+        case CQT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CQT_ERR_CUDA: return "CUDA error";
+        case CQT_ERR_STATE: return "call not valid in this state";
+        case CQT_ERR_DEVICE_CHECK: return "device-side check failed";
+    }
+    return "unknown status";
+}
+
+cqt_status cqt_plan_create(double fs, double fmin, double fmax, int bins_per_octave, int64_t L, cqt_window window,
+                           cqt_plan **out) {
+    cqt_plan_desc d;
+    d.fs = fs; d.fmin = fmin; d.fmax = fmax; d.bins_per_octave = bins_per_octave; d.L = L;
+    d.window = (int)window; d.m_policy = CQT_M_MULT4; d.min_win = 4.0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return CQT_ERR_CUDA;
+    d.device = dev;
+    return cqt_plan_create_ex(&d, out);
+}
+
+cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
+    if (!desc || !out) return CQT_ERR_INVALID_ARG;
+    const int64_t N = desc->L;
+    if (N < 0) return CQT_ERR_INVALID_ARG;
+    if (!is_pow2(N) || N < 64 || N > (1ll << 22)) return CQT_ERR_UNSUPPORTED;
+    cqt_plan *p = new (std::nothrow) cqt_plan();
+    if (!p) return CQT_ERR_CUDA;
+    LayoutDesc ld{desc->fs, desc->fmin, desc->fmax, desc->bins_per_octave, N, desc->window, desc->m_policy,
+                  desc->min_win > 0 ? desc->min_win : 4.0};
+    std::string why;
+    int rc = build_layout(ld, p->lay, why);
+    if (rc != 0) { delete p; return (cqt_status)rc; }
+    p->N = N;
+    p->device = desc->device;
+    const HostLayout &L = p->lay;
+    p->g32.resize(L.table_len);
+    p->h32.resize(L.table_len);
+    for (int64_t i = 0; i < L.table_len; ++i) { p->g32[i] = (float)L.g[i]; p->h32[i] = (float)L.h[i]; }
+    p->y_pitch = (L.y_len + 7) / 8 * 8;
+
+    // ---- transform-length plans and twiddles
+    std::vector<float2> tw;
+    std::map<int64_t, int> fft_of;
+    auto plan_for = [&](int64_t M, bool pow2) -> int {
+        const int64_t key = pow2 ? -M : M;
+        auto it = fft_of.find(key);
+        if (it != fft_of.end()) return it->second;
+        FftPlan fp;
+        if (!make_fft_plan(M, pow2, tw, fp)) return -1;
+        p->ffts.push_back(fp);
+        return fft_of[key] = (int)p->ffts.size() - 1;
+    };
+    LongFft &lf = p->lf;
+    lf.Lp = N / 2;
+    if (lf.Lp <= 16384) { lf.A = 1; lf.B = lf.Lp; }
+    else {
+        int lg = 0;
+        while ((1ll << lg) < lf.Lp) ++lg;
+        lf.B = std::min<int64_t>(1024, 1ll << ((lg + 1) / 2));
+        lf.A = lf.Lp / lf.B;
+    }
+    lf.fft_B = plan_for(lf.B, true);
+    lf.fft_A = lf.A > 1 ? plan_for(lf.A, true) : lf.fft_B;
+    lf.tw_lp = append_twiddles(tw, lf.Lp, lf.log_lp_c);
+    lf.tw_n = append_twiddles(tw, N, lf.log_n_c);
+    lf.tw_rows = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.B <= 512 ? 16 : 8, lf.A / 2);
+    lf.tw_cols = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.A <= 1024 ? 16 : 8, lf.B);
+    lf.x_pitch = (lf.Lp + 1 + 7) / 8 * 8;
+
+    // ---- band records
+    p->bands.resize(L.bands.size());
+    for (size_t i = 0; i < L.bands.size(); ++i) {
+        const HostBand &hb = L.bands[i];
+        BandRec &br = p->bands[i];
+        br.kc = (int32_t)hb.kc; br.d0 = (int32_t)hb.d0; br.S = (int32_t)hb.S; br.M = (int32_t)hb.M;
+        br.tab_off = (int32_t)hb.tab_off; br.coeff_off = (int32_t)hb.coeff_off; br.y_off = (int32_t)hb.y_off;
+        br.j_lo = (int32_t)hb.j_lo; br.n_in = (int32_t)hb.n_in; br.side = hb.side;
+        br.inv_M = (float)(1.0 / (double)hb.M);
+        br.fft = plan_for(hb.M, false);
+        if (br.fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
+    }
+    // ---- launch classes by band length
+    const int limits[kNumClasses] = {128, 2048, 8192, 1 << 30};
+    const int threads[kNumClasses] = {256, 128, 256, 512};
+    for (int c = 0; c < kNumClasses; ++c) {
+        p->cls[c].threads = threads[c];
+        p->cls[c].items_per_cta = c == 0 ? 8 : 1;
+    }
+    std::vector<int> order(L.bands.size());
+    for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L.bands[a].M > L.bands[b].M; });
+    const int64_t smem_cap_elems = (227 * 1024) / 8;
+    for (int i : order) {
+        const int64_t M = L.bands[i].M;
+        const int64_t elems = p->ffts[p->bands[i].fft].generic ? 2 * M : M;
+        int c = 0;
+        while (M > limits[c]) ++c;
+        if (elems * p->cls[c].items_per_cta > smem_cap_elems) { delete p; return CQT_ERR_UNSUPPORTED; }
+        p->cls[c].work.push_back(i);
+        p->cls[c].max_elems = (int)std::max<int64_t>(p->cls[c].max_elems, elems);
+        p->cls[c].n_bands++;
+    }
+    if (p->device < 0) { *out = p; return CQT_OK; }
+
+    // ---- device tables
+    int cur = 0;
+    if (cudaGetDevice(&cur) != cudaSuccess || cudaSetDevice(p->device) != cudaSuccess) { p->device = -1; delete p; return CQT_ERR_CUDA; }
+    std::vector<float> tA(L.table_len), tS(L.table_len), tTA(L.table_len), tSA(L.table_len);
+    std::vector<int2> span(L.bands.size());
+    for (size_t i = 0; i < L.bands.size(); ++i) {
+        const HostBand &hb = L.bands[i];
+        span[i] = make_int2((int)(hb.kc + hb.d0 + hb.j_lo), (int)hb.y_off);
+        for (int64_t j = 0; j < hb.S; ++j) {
+            const int64_t k = hb.kc + hb.d0 + j;
+            const double g = L.g[hb.tab_off + j], h = L.h[hb.tab_off + j];
+            const double wk = (k == 0 || k == N / 2) ? 1.0 : 2.0;
+            tA[hb.tab_off + j] = (float)(g / (double)hb.M);
+            tS[hb.tab_off + j] = (float)h;
+            tTA[hb.tab_off + j] = (float)((double)N * g / (2.0 * (double)hb.M));
+            tSA[hb.tab_off + j] = (float)(h * wk / (double)N);
+        }
+    }
+    std::vector<int32_t> cover(N / 2 + 1);
+    for (int64_t k = 0; k <= N / 2; ++k) cover[k] = (L.cover_lo[k] << 8) | L.cover_n[k];
+    cudaError_t e = cudaSuccess;
+    auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+    chk(upload(p->d.bands, p->bands));
+    chk(upload(p->d.ffts, p->ffts));
+    chk(upload(p->d.tw, tw));
+    chk(upload(p->d.tab_analysis, tA));
+    chk(upload(p->d.tab_synthesis, tS));
+    chk(upload(p->d.tab_analysis_adj, tTA));
+    chk(upload(p->d.tab_synthesis_adj, tSA));
+    chk(upload(p->d.cover, cover));
+    chk(upload(p->d.span, span));
+    for (auto &c : p->cls) chk(upload(c.d_work, c.work));
+    cudaDeviceProp prop;
+    chk(cudaGetDeviceProperties(&prop, p->device));
+    p->sm_count = prop.multiProcessorCount;
+    p->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    if (e == cudaSuccess) chk(configure_band_kernels(*p));
+    if (e == cudaSuccess) chk(configure_long_fft_kernels(*p));
+    cudaSetDevice(cur);
+    if (e != cudaSuccess) { cqt_plan_destroy(p); return CQT_ERR_CUDA; }
+    *out = p;
+    return CQT_OK;
+}
+
+cqt_status cqt_plan_destroy(cqt_plan *p) {
+    if (!p) return CQT_OK;
+    free_device(p);
+    delete p;
+    return CQT_OK;
+}
+
+int64_t cqt_plan_num_bands(const cqt_plan *p) { return p ? (int64_t)p->lay.bands.size() : -1; }
+int64_t cqt_plan_coeff_count(const cqt_plan *p) { return p ? p->lay.coeff_count : -1; }
+int64_t cqt_plan_signal_length(const cqt_plan *p) { return p ? p->N : -1; }
+int64_t cqt_plan_table_length(const cqt_plan *p) { return p ? p->lay.table_len : -1; }
+
+cqt_status cqt_plan_band_info(const cqt_plan *p, int64_t band, cqt_band_info *out) {
+    if (!p || !out || band < 0 || band >= (int64_t)p->lay.bands.size()) return CQT_ERR_INVALID_ARG;
+    const HostBand &hb = p->lay.bands[band];
+    out->centre_hz = hb.centre_hz; out->centre_bin = hb.kc; out->support = hb.S; out->first_offset = hb.d0;
+    out->M = hb.M; out->coeff_offset = hb.coeff_off; out->table_offset = hb.tab_off; out->is_sideband = hb.side;
+    return CQT_OK;
+}
+
+size_t cqt_plan_workspace_bytes(const cqt_plan *p, int64_t batch) {
+    if (!p || batch <= 0) return 0;
+    const int64_t t = p->lf.A > 1 ? p->lf.Lp : 0;
+    const int64_t per = std::max<int64_t>(t + p->lf.x_pitch, t + p->y_pitch);
+    return (size_t)(256 + batch * per * (int64_t)sizeof(float2));
+}
+
+cqt_status cqt_plan_tables(const cqt_plan *p, const float **g_host, const float **h_host) {
+    if (!p) return CQT_ERR_INVALID_ARG;
+    if (g_host) *g_host = p->g32.data();
+    if (h_host) *h_host = p->h32.data();
+    return CQT_OK;
+}
+
+cqt_status cqt_plan_check(const cqt_plan *p) { return p ? CQT_OK : CQT_ERR_INVALID_ARG; }
+
+}  // extern "C"
+
+namespace {
+
+struct Call {
+    const cqt_plan *p;
+    float2 *T, *second;   // workspace regions
+    cudaStream_t st;
+    int prev_dev;
+};
+
+cqt_status begin_call(const cqt_plan *p, const void *sig, int64_t stride, int64_t batch, int64_t valid_len,
+                      const void *coef, void *ws, size_t ws_bytes, void *stream, Call &c) {
+    if (!p || !sig || !coef) return CQT_ERR_INVALID_ARG;
+    if (batch <= 0 || batch > 65535 || valid_len <= 0 || valid_len > p->N || stride < valid_len) return CQT_ERR_INVALID_ARG;
+    if (p->device < 0) return CQT_ERR_STATE;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) || ws_bytes < cqt_plan_workspace_bytes(p, batch)) return CQT_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(coef) & 7) || (reinterpret_cast<uintptr_t>(sig) & 3)) return CQT_ERR_INVALID_ARG;
+    c.p = p;
+    c.T = reinterpret_cast<float2 *>(ws);
+    c.second = c.T + (p->lf.A > 1 ? batch * p->lf.Lp : 0);
+    c.st = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaGetDevice(&c.prev_dev) != cudaSuccess) return CQT_ERR_CUDA;
+    if (c.prev_dev != p->device && cudaSetDevice(p->device) != cudaSuccess) return CQT_ERR_CUDA;
+    return CQT_OK;
+}
+
+cqt_status end_call(const Call &c, cudaError_t e) {
+    if (c.prev_dev != c.p->device) cudaSetDevice(c.prev_dev);
+    return e == cudaSuccess ? CQT_OK : CQT_ERR_CUDA;
+}
+
+cqt_status run_analysis_form(const cqt_plan *p, const float *table, const float *x, int64_t x_stride, int64_t batch,
+                             int64_t valid_len, cqt_c64 *c, void *ws, size_t ws_bytes, void *stream) {
+    Call k;
+    cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
+    if (s != CQT_OK) return s;
+    cudaError_t e = launch_rfft_forward(*p, x, x_stride, batch, valid_len, k.T, k.second, k.st);
+    if (e == cudaSuccess) e = launch_bands_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), batch, k.st);
+    return end_call(k, e);
+}
+
+cqt_status run_synthesis_form(const cqt_plan *p, const float *table, bool fold, const cqt_c64 *c, int64_t batch,
+                              int64_t valid_len, float *x, int64_t x_stride, void *ws, size_t ws_bytes, void *stream) {
+    Call k;
+    cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
+    if (s != CQT_OK) return s;
+    cudaError_t e = launch_bands_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, batch, k.st);
+    if (e == cudaSuccess) e = launch_rfft_inverse(*p, k.second, k.T, x, x_stride, batch, valid_len, k.st);
+    return end_call(k, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+cqt_status cqt_analyse(const cqt_plan *p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,
+                       cqt_c64 *c, void *ws, size_t ws_bytes, void *stream) {
+    return run_analysis_form(p, p ? p->d.tab_analysis : nullptr, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream);
+}
+
+cqt_status cqt_synthesise(const cqt_plan *p, const cqt_c64 *c, int64_t batch, int64_t valid_len, float *x,
+                          int64_t x_stride, void *ws, size_t ws_bytes, void *stream) {
+    return run_synthesis_form(p, p ? p->d.tab_synthesis : nullptr, false, c, batch, valid_len, x, x_stride, ws, ws_bytes, stream);
+}
+
+cqt_status cqt_analyse_adjoint(const cqt_plan *p, const cqt_c64 *c_bar, int64_t batch, int64_t valid_len, float *x_bar,
+                               int64_t x_stride, void *ws, size_t ws_bytes, void *stream) {
+    return run_synthesis_form(p, p ? p->d.tab_analysis_adj : nullptr, true, c_bar, batch, valid_len, x_bar, x_stride, ws, ws_bytes, stream);
+}
+
+cqt_status cqt_synthesise_adjoint(const cqt_plan *p, const float *x_bar, int64_t x_stride, int64_t batch,
+                                  int64_t valid_len, cqt_c64 *c_bar, void *ws, size_t ws_bytes, void *stream) {
+    return run_analysis_form(p, p ? p->d.tab_synthesis_adj : nullptr, x_bar, x_stride, batch, valid_len, c_bar, ws, ws_bytes, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+// Internal interfaces between the plan builder, the kernel launchers and the C ABI.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "layout.hpp"
+#include "plan_types.h"
+
+namespace cqt {
+
+constexpr int kNumClasses = 4;
+
+// Launch shape of one band-length class.
+struct BandClass {
+    int threads = 0;         // threads per CTA
+    int items_per_cta = 1;   // > 1: one warp per (band, signal) item
+    int max_elems = 0;       // shared-memory elements (float2) per item
+    int n_bands = 0;         // bands in the class
+    int32_t *d_work = nullptr;  // band indices, longest first
+    std::vector<int32_t> work;
+};
+
+struct LongFft {
+    int64_t Lp = 0, A = 1, B = 0;
+    int fft_A = -1, fft_B = -1;   // FftPlan indices
+    int tw_lp = 0, tw_n = 0;      // two-level tables of W_Lp and W_N inside the twiddle array
+    int log_lp_c = 0, log_n_c = 0;
+    int tw_rows = 1;              // rows per mirrored half handled by one CTA of the row kernels
+    int tw_cols = 1;              // columns per CTA of the column kernels
+    int64_t x_pitch = 0;          // elements per signal of the half-spectrum buffer (Lp + 1 rounded up)
+};
+
+struct DevicePlan {
+    BandRec *bands = nullptr;
+    FftPlan *ffts = nullptr;
+    float2 *tw = nullptr;
+    float *tab_analysis = nullptr;     // g / M
+    float *tab_synthesis = nullptr;    // h
+    float *tab_analysis_adj = nullptr; // N g / (2 M)
+    float *tab_synthesis_adj = nullptr;// h w_k / N
+    int32_t *cover = nullptr;          // per bin: (first covering band << 8) | count
+    int2 *span = nullptr;              // per band: (first in-range bin, offset in the weighted-bin row)
+};
+
+}  // namespace cqt
+
+struct cqt_plan {
+    cqt::HostLayout lay;
+    std::vector<float> g32, h32;
+    std::vector<cqt::FftPlan> ffts;
+    std::vector<cqt::BandRec> bands;
+    int device = -1;
+    int64_t N = 0;
+    int64_t y_pitch = 0;
+    cqt::LongFft lf;
+    cqt::BandClass cls[cqt::kNumClasses];
+    cqt::DevicePlan d;
+    int max_smem_optin = 0;
+    int sm_count = 0;
+};
+
+namespace cqt {
+
+// table selectors of the band kernels
+enum { TAB_ANALYSIS = 0, TAB_SYNTHESIS = 1, TAB_ANALYSIS_ADJ = 2, TAB_SYNTHESIS_ADJ = 3 };
+
+// long_fft.cu
+cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,
+                                float2 *T, float2 *X, cudaStream_t st);
+cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, float *x, int64_t x_stride,
+                                int64_t batch, int64_t valid_len, cudaStream_t st);
+cudaError_t configure_long_fft_kernels(const cqt_plan &p);
+
+// band.cu
+cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
+                                       int64_t batch, cudaStream_t st);
+cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool fold_sidebands, const float2 *c,
+                                     float2 *Y, int64_t batch, cudaStream_t st);
+cudaError_t configure_band_kernels(const cqt_plan &p);
+
+}  // namespace cqt

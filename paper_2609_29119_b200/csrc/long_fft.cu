@@ -1,0 +1,346 @@
+// Packed real FFT of length N through a complex FFT of length Lp = N/2 = A * B (Eq. pack), with
+// the conjugate-symmetric fold (Eq. untangle) in the epilogue of the last forward pass and the
+// inverse fold (Eq. retangle) plus the deterministic per-bin sum over bands in the prologue of the
+// first inverse pass.
+//
+// Index split:  sample index j = j1 * B + j2,  bin index k = k1 + A * k2  (j1,k1 < A; j2,k2 < B).
+//   forward  pass C ("columns"): for TWc adjacent j2, A-point DFT over j1, times W_Lp^{j2 k1},
+//                                written to T[k1][j2].
+//            pass R ("rows"):    for a set of rows k1, B-point DFT over j2 gives Z[k1 + A k2];
+//                                a CTA owns TWr rows and their mirror images A - k1 (plus one
+//                                extra row each side) so both operands of Eq. untangle are in its
+//                                shared memory; writes the half spectrum X[0 .. Lp].
+//   inverse  pass R':            gathers X^_q = sum over covering bands (fixed order), forms Z_q by
+//                                Eq. retangle, inverse B-point DFT over q2, times conj W_Lp^{j2 q1},
+//                                written to T[q1][j2].
+//            pass C':            inverse A-point DFT over q1, scaled, unpacked to x[2j], x[2j+1].
+// When Lp is small (A == 1) the row kernels read / write the signal directly and passes C, C' vanish.
+#include "engine.cuh"
+#include "internal.hpp"
+
+namespace cqt {
+
+extern __shared__ float2 smem_long[];
+
+struct LongArgs {
+    const FftPlan *ffts;
+    const float2 *tw;
+    int fft_A, fft_B;
+    int A, B, Lp;
+    int tw_lp, log_lp_c;   // two-level table of W_Lp
+    int tw_n, log_n_c;     // two-level table of W_N
+    int tw_cols, tw_rows;
+    int valid_len;
+    int aligned;           // signal rows allow float2 access
+    long long x_stride;
+    const float *x_in;
+    float *x_out;
+    float2 *T;
+    long long t_pitch;
+    float2 *X;             // half spectrum rows (forward)
+    long long x_pitch;
+    // inverse gather
+    const float2 *Y;
+    long long y_pitch;
+    const int32_t *cover;
+    const int2 *span;
+    float scale;
+    uint32_t cols_magic, rows_magic;
+};
+
+__device__ __forceinline__ float2 load_packed(const float *row, long long j, int valid_len, int aligned) {
+    const long long i = 2 * j;
+    if (i + 1 < valid_len) {
+        if (aligned) return __ldg(reinterpret_cast<const float2 *>(row + i));
+        return make_float2(__ldg(row + i), __ldg(row + i + 1));
+    }
+    if (i < valid_len) return make_float2(__ldg(row + i), 0.f);
+    return make_float2(0.f, 0.f);
+}
+
+__device__ __forceinline__ void store_packed(float *row, long long j, float2 v, int valid_len, int aligned) {
+    const long long i = 2 * j;
+    if (i + 1 < valid_len) {
+        if (aligned) *reinterpret_cast<float2 *>(row + i) = v;
+        else { row[i] = v.x; row[i + 1] = v.y; }
+    } else if (i < valid_len) {
+        row[i] = v.x;
+    }
+}
+
+// ---------------------------------------------------------------- forward, pass C
+__global__ void __launch_bounds__(512) rfft_cols_fwd_kernel(LongArgs a) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int TW = a.tw_cols;
+    const int j2_0 = blockIdx.x * TW;
+    const int ch = blockIdx.y;
+    const FftPlan &fp = a.ffts[a.fft_A];
+    float2 *buf = smem_long;
+    const float *row = a.x_in + (long long)ch * a.x_stride;
+    const int total = a.A * TW;
+    for (int e = tid; e < total; e += nthr) {
+        const int j1 = e / TW, c = e - j1 * TW;
+        buf[e] = load_packed(row, (long long)j1 * a.B + j2_0 + c, a.valid_len, a.aligned);
+    }
+    __syncthreads();
+    fft_dif<-1, BlockSync, true>(buf, nullptr, TW, TW, a.cols_magic, fp, a.tw, tid, nthr);
+    float2 *T = a.T + (long long)ch * a.t_pitch;
+    const float2 *wl = a.tw + a.tw_lp;
+    for (int e = tid; e < total; e += nthr) {
+        const int k1 = e / TW, c = e - k1 * TW;
+        const float2 v = buf[dif_pos(fp, k1) * TW + c];
+        const float2 w = twiddle(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
+        T[(long long)k1 * a.B + j2_0 + c] = cmul(v, w);
+    }
+}
+
+// rows owned by CTA t of the row kernels: first set TWr*t + i, second set A - TWr*t - TWr + i
+// (i < TWr owned; i == TWr is the extra, read-only row of each set; row A means row 0)
+__device__ __forceinline__ int row_of(int t, int r, int TW, int A) {
+    const int i = r <= TW ? r : r - (TW + 1);
+    const int k1 = r <= TW ? TW * t + i : A - TW * t - TW + i;
+    return k1 >= A ? k1 - A : k1;
+}
+
+// ---------------------------------------------------------------- forward, pass R (+ untangle)
+__global__ void __launch_bounds__(512) rfft_rows_fwd_kernel(LongArgs a) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int ch = blockIdx.y, t = blockIdx.x;
+    const int A = a.A, B = a.B, TW = a.tw_rows;
+    const bool direct = (A == 1);
+    const int ncols = direct ? 1 : 2 * TW + 2;
+    const int pitch = direct ? 1 : ncols + 1;   // odd: the transposing load is conflict-free
+    const FftPlan &fp = a.ffts[a.fft_B];
+    float2 *buf = smem_long;
+    if (direct) {
+        const float *row = a.x_in + (long long)ch * a.x_stride;
+        for (int e = tid; e < B; e += nthr) buf[e] = load_packed(row, e, a.valid_len, a.aligned);
+    } else {
+        const float2 *T = a.T + (long long)ch * a.t_pitch;
+        for (int e = tid; e < ncols * B; e += nthr) {
+            const int r = e / B, j2 = e - r * B;
+            buf[(size_t)j2 * pitch + r] = __ldg(T + (long long)row_of(t, r, TW, A) * B + j2);
+        }
+    }
+    __syncthreads();
+    fft_dif<-1, BlockSync, true>(buf, nullptr, pitch, ncols, a.rows_magic, fp, a.tw, tid, nthr);
+    float2 *X = a.X + (long long)ch * a.x_pitch;
+    const float2 *wn = a.tw + a.tw_n;
+    const int nown = direct ? 1 : 2 * TW;
+    for (int e = tid; e < nown * B; e += nthr) {
+        const int k2 = e / nown, o = e - k2 * nown;
+        // owned row o -> column index r in shared memory, and the partner's column / k2
+        int r, rp, k2p;
+        if (direct) {
+            r = 0; rp = 0; k2p = k2 == 0 ? 0 : B - k2;
+        } else {
+            r = o < TW ? o : o + 1;                      // skip the extra row of the first set
+            const int i = o < TW ? o : o - TW;
+            rp = o < TW ? (TW + 1) + (TW - i) : (TW - i);   // mirror row's column
+            k2p = B - 1 - k2;
+        }
+        const int k1 = direct ? 0 : row_of(t, r, TW, A);
+        if (!direct && k1 == 0) { rp = r; k2p = k2 == 0 ? 0 : B - k2; }
+        const float2 z = buf[(size_t)dif_pos(fp, k2) * pitch + r];
+        const float2 zp = buf[(size_t)dif_pos(fp, k2p) * pitch + rp];
+        const int k = k1 + A * k2;
+        // X_k = 1/2 (1 - i w) Z_k + 1/2 (1 + i w) conj Z_{Lp-k},  w = exp(-2 pi i k / N)
+        const float2 w = twiddle(wn, a.log_n_c, (uint32_t)k);
+        const float2 ev = make_float2(0.5f * (z.x + zp.x), 0.5f * (z.y - zp.y));   // (Z + conj Zp)/2
+        const float2 od = make_float2(0.5f * (z.x - zp.x), 0.5f * (z.y + zp.y));   // (Z - conj Zp)/2
+        // -i w od = (w.y od.x + w.x od.y) + i (w.y od.y - w.x od.x)
+        const float2 xk = make_float2(ev.x + (w.y * od.x + w.x * od.y), ev.y + (w.y * od.y - w.x * od.x));
+        X[k] = xk;
+        if (k == 0) X[a.Lp] = make_float2(z.x - z.y, 0.f);
+    }
+}
+
+// ---------------------------------------------------------------- inverse, pass R' (gather + retangle)
+__device__ __forceinline__ float2 gather_bin(const float2 *__restrict__ Y, const int32_t *__restrict__ cover,
+                                             const int2 *__restrict__ span, int k) {
+    const int32_t cv = __ldg(cover + k);
+    const int lo = cv >> 8, n = cv & 255;
+    float2 acc = make_float2(0.f, 0.f);
+    for (int i = 0; i < n; ++i) {
+        const int2 sp = __ldg(span + lo + i);
+        const float2 v = __ldg(Y + sp.y + (k - sp.x));
+        acc.x += v.x;
+        acc.y += v.y;
+    }
+    return acc;
+}
+
+__global__ void __launch_bounds__(512) irfft_rows_kernel(LongArgs a) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int ch = blockIdx.y, t = blockIdx.x;
+    const int A = a.A, B = a.B, TW = a.tw_rows, Lp = a.Lp;
+    const bool direct = (A == 1);
+    const int ncols = direct ? 1 : TW;
+    const int pitch = direct ? 1 : (TW | 1);
+    const FftPlan &fp = a.ffts[a.fft_B];
+    float2 *buf = smem_long;
+    const float2 *Y = a.Y + (long long)ch * a.y_pitch;
+    const float2 *wn = a.tw + a.tw_n;
+    for (int e = tid; e < ncols * B; e += nthr) {
+        const int q2 = e / ncols, r = e - q2 * ncols;
+        const int q1 = direct ? 0 : t * TW + r;
+        const int q = q1 + A * q2;
+        float2 xq = gather_bin(Y, a.cover, a.span, q);
+        float2 xm = gather_bin(Y, a.cover, a.span, Lp - q);
+        if (q == 0) { xq.y = 0.f; xm.y = 0.f; }   // bins 0 and N/2 are made real
+        // Z_q = 1/2 [(1 + i conj w) X_q + (1 - i conj w) conj X_{Lp-q}],  w = exp(-2 pi i q / N)
+        const float2 w = twiddle(wn, a.log_n_c, (uint32_t)q);
+        const float2 ev = make_float2(xq.x + xm.x, xq.y - xm.y);   // X_q + conj X_m
+        const float2 od = make_float2(xq.x - xm.x, xq.y + xm.y);   // X_q - conj X_m
+        // i conj(w) od = i (w.x - i w.y)... conj w = (w.x, -w.y); i*conj w = (w.y, w.x)
+        const float2 icw = make_float2(w.y, w.x);
+        const float2 rot = cmul(icw, od);
+        buf[(size_t)q2 * pitch + r] = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
+    }
+    __syncthreads();
+    fft_dif<+1, BlockSync, true>(buf, nullptr, pitch, ncols, a.rows_magic, fp, a.tw, tid, nthr);
+    if (direct) {
+        float *row = a.x_out + (long long)ch * a.x_stride;
+        for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[dif_pos(fp, j)], a.valid_len, a.aligned);
+    } else {
+        float2 *T = a.T + (long long)ch * a.t_pitch;
+        const float2 *wl = a.tw + a.tw_lp;
+        for (int e = tid; e < ncols * B; e += nthr) {
+            const int r = e / B, j2 = e - r * B;
+            const int q1 = t * TW + r;
+            const float2 v = buf[(size_t)dif_pos(fp, j2) * pitch + r];
+            const float2 w = cconj(twiddle(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
+            T[(long long)q1 * B + j2] = cmul(v, w);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- inverse, pass C' (+ unpack)
+__global__ void __launch_bounds__(512) irfft_cols_kernel(LongArgs a) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int TW = a.tw_cols;
+    const int j2_0 = blockIdx.x * TW;
+    const int ch = blockIdx.y;
+    const FftPlan &fp = a.ffts[a.fft_A];
+    float2 *buf = smem_long;
+    const float2 *T = a.T + (long long)ch * a.t_pitch;
+    const int total = a.A * TW;
+    for (int e = tid; e < total; e += nthr) {
+        const int q1 = e / TW, c = e - q1 * TW;
+        buf[e] = __ldg(T + (long long)q1 * a.B + j2_0 + c);
+    }
+    __syncthreads();
+    fft_dif<+1, BlockSync, true>(buf, nullptr, TW, TW, a.cols_magic, fp, a.tw, tid, nthr);
+    float *row = a.x_out + (long long)ch * a.x_stride;
+    for (int e = tid; e < total; e += nthr) {
+        const int j1 = e / TW, c = e - j1 * TW;
+        store_packed(row, (long long)j1 * a.B + j2_0 + c, buf[dif_pos(fp, j1) * TW + c], a.valid_len, a.aligned);
+    }
+}
+
+// ---------------------------------------------------------------- host side
+static uint32_t magic_of(uint32_t d) { return d <= 1 ? 0u : (uint32_t)(((1ull << 32) + d - 1) / d); }
+
+static LongArgs base_args(const cqt_plan &p, int64_t valid_len, int64_t x_stride, const void *xptr) {
+    LongArgs a{};
+    a.ffts = p.d.ffts;
+    a.tw = p.d.tw;
+    a.fft_A = p.lf.fft_A;
+    a.fft_B = p.lf.fft_B;
+    a.A = (int)p.lf.A;
+    a.B = (int)p.lf.B;
+    a.Lp = (int)p.lf.Lp;
+    a.tw_lp = p.lf.tw_lp;
+    a.log_lp_c = p.lf.log_lp_c;
+    a.tw_n = p.lf.tw_n;
+    a.log_n_c = p.lf.log_n_c;
+    a.tw_cols = p.lf.tw_cols;
+    a.tw_rows = p.lf.tw_rows;
+    a.valid_len = (int)valid_len;
+    a.x_stride = x_stride;
+    a.aligned = ((reinterpret_cast<uintptr_t>(xptr) & 7) == 0 && (x_stride & 1) == 0) ? 1 : 0;
+    a.t_pitch = p.lf.Lp;
+    a.x_pitch = p.lf.x_pitch;
+    a.y_pitch = p.y_pitch;
+    a.cover = p.d.cover;
+    a.span = p.d.span;
+    a.cols_magic = magic_of(a.tw_cols);
+    return a;
+}
+
+static size_t rows_fwd_smem(const LongFft &lf) {
+    return lf.A == 1 ? (size_t)lf.B * 8 : (size_t)lf.B * (2 * lf.tw_rows + 3) * 8;
+}
+static size_t rows_inv_smem(const LongFft &lf) {
+    return lf.A == 1 ? (size_t)lf.B * 8 : (size_t)lf.B * (lf.tw_rows | 1) * 8;
+}
+static size_t cols_smem(const LongFft &lf) { return (size_t)lf.A * lf.tw_cols * 8; }
+
+static int threads_for(size_t butterflies) {
+    int t = 64;
+    while (t < 512 && (size_t)t < butterflies) t *= 2;
+    return t;
+}
+
+cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,
+                                float2 *T, float2 *X, cudaStream_t st) {
+    LongArgs a = base_args(p, valid_len, x_stride, x);
+    a.x_in = x;
+    a.T = T;
+    a.X = X;
+    const LongFft &lf = p.lf;
+    if (lf.A > 1) {
+        dim3 grid((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
+        rfft_cols_fwd_kernel<<<grid, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(lf), st>>>(a);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        a.rows_magic = magic_of(2 * lf.tw_rows + 2);
+        dim3 grid2((unsigned)(lf.A / (2 * lf.tw_rows)), (unsigned)batch);
+        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows + 2) / 8), rows_fwd_smem(lf), st>>>(a);
+    } else {
+        a.rows_magic = 0;
+        dim3 grid2(1, (unsigned)batch);
+        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B / 8), rows_fwd_smem(lf), st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, float *x, int64_t x_stride,
+                                int64_t batch, int64_t valid_len, cudaStream_t st) {
+    LongArgs a = base_args(p, valid_len, x_stride, x);
+    a.x_out = x;
+    a.T = T;
+    a.Y = Y;
+    a.scale = (float)(0.5 / (double)p.lf.Lp);
+    const LongFft &lf = p.lf;
+    if (lf.A > 1) {
+        a.rows_magic = magic_of(lf.tw_rows);
+        dim3 grid((unsigned)(lf.A / lf.tw_rows), (unsigned)batch);
+        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B * lf.tw_rows / 8), rows_inv_smem(lf), st>>>(a);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        dim3 grid2((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
+        irfft_cols_kernel<<<grid2, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(lf), st>>>(a);
+    } else {
+        a.rows_magic = 0;
+        dim3 grid(1, (unsigned)batch);
+        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B / 8), rows_inv_smem(lf), st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t configure_long_fft_kernels(const cqt_plan &p) {
+    cudaError_t e;
+    e = cudaFuncSetAttribute(rfft_rows_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_fwd_smem(p.lf));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(irfft_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_inv_smem(p.lf));
+    if (e != cudaSuccess) return e;
+    if (p.lf.A > 1) {
+        e = cudaFuncSetAttribute(rfft_cols_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p.lf));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(irfft_cols_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p.lf));
+    }
+    return e;
+}
+
+}  // namespace cqt

@@ -1,0 +1,50 @@
+// Structures shared by the host plan builder and the kernels (plain data, no CUDA types).
+#pragma once
+#include <stdint.h>
+
+namespace cqt {
+
+constexpr int kMaxStages = 8;
+
+// In-place decimation-in-frequency plan of one transform length M = r_1 r_2 ... r_d.
+// Stage j works on sub-transforms of length n_j = M / (r_1 .. r_{j-1}) with butterfly stride
+// s_j = n_j / r_j.  Frequency k = k_1 + r_1 (k_2 + r_2 (...)) ends at position
+// ((k_1 r_2 + k_2) r_3 + ...) (mixed-radix digit reversal).
+// Twiddles exp(-2 pi i y / M) are the product of two table entries:
+//   tw[tw_off + (y & (C-1))] * tw[tw_off + C + (y >> logC)],  C = 1 << logC.
+struct FftPlan {
+    int32_t M;
+    int32_t nstages;
+    int32_t logC;
+    int32_t tw_off;                 // into the plan's twiddle array (float2 elements)
+    int32_t generic;                // 1 if stage 0 is a generic (out-of-place) radix
+    int32_t pad_[3];
+    int32_t radix[kMaxStages];
+    int32_t stride[kMaxStages];     // s_j
+    uint32_t rmagic[kMaxStages];    // ceil(2^32 / r_j)
+    uint32_t smagic[kMaxStages];    // ceil(2^32 / s_j)
+};
+
+// One band of the layout as the kernels see it.
+struct BandRec {
+    int32_t kc;         // centre bin
+    int32_t d0;         // first (most negative) support offset
+    int32_t S;          // support size
+    int32_t M;          // coefficients
+    int32_t tab_off;    // into the window tables (S entries, offset order)
+    int32_t coeff_off;  // into one signal's coefficient row
+    int32_t y_off;      // into one signal's weighted-bin scratch row (in-range entries only)
+    int32_t j_lo;       // first support index whose bin lies in 0..N/2
+    int32_t n_in;       // number of support entries whose bin lies in 0..N/2
+    int32_t side;       // 0 regular, 1 DC, 2 Nyquist
+    int32_t fft;        // index of the FftPlan for M
+    float inv_M;
+};
+
+// Per-bin cover: bands cover_lo .. cover_lo + cover_n - 1 contain the bin (contiguous because
+// support starts and ends are monotone in the band index).
+struct BinCover {
+    int32_t lo_n;       // (cover_lo << 8) | cover_n
+};
+
+}  // namespace cqt

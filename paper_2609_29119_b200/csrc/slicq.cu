@@ -1,0 +1,249 @@
+// Sliced streaming form (Sec. 4, slicing paragraph): slices of sl samples with hop sl/2 and a
+// Tukey transition window, each analysed and synthesised independently, reconstructions
+// overlap-added in slice order.  All bookkeeping is host-side integer arithmetic; device work is
+// enqueued on the caller's stream and never synchronised here.
+#include <algorithm>
+#include <cmath>
+#include <new>
+#include <vector>
+
+#include "../../include/cqt.h"
+#include "internal.hpp"
+
+struct cqt_slicq {
+    const cqt_plan *plan = nullptr;
+    int C = 0;
+    int64_t sl = 0, H = 0, tr = 0, K = 0;
+    int64_t ring_in = 0, ring_out = 0;   // samples per channel
+    float *d_win = nullptr;              // [sl]
+    float *d_in = nullptr;               // [C][ring_in], stream sample n at n mod ring_in
+    float *d_stage = nullptr;            // [K*C][sl] windowed slices / reconstructed slices
+    cqt_c64 *d_coef = nullptr;           // [K][C][coeff_count]
+    float *d_out = nullptr;              // [C][ring_out], output sample n at n mod ring_out
+    void *d_ws = nullptr;
+    size_t ws_bytes = 0, total_bytes = 0;
+    int64_t n_in = 0;        // frames pushed
+    int64_t next_slice = 0;  // first slice not yet analysed
+    int64_t next_synth = 0;  // first slice not yet synthesised
+    int64_t n_out = 0;       // frames pulled
+};
+
+namespace {
+
+__global__ void slicq_ingest_kernel(const float *x, long long x_stride, float *ring, long long R, long long pos, long long n, int zero) {
+    const int c = blockIdx.y;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        ring[c * R + (pos + i) % R] = zero ? 0.f : x[c * x_stride + i];
+}
+
+// stage[(s - s0) * C + c][i] = w[i] * stream[c][s H - H + i]  (zero before the start of the stream)
+__global__ void slicq_cut_kernel(const float *ring, long long R, const float *w, float *stage, long long sl, long long H,
+                                 long long s0, int C) {
+    const long long s = s0 + blockIdx.y / C;
+    const int c = blockIdx.y % C;
+    float *dst = stage + (long long)blockIdx.y * sl;
+    const long long first = s * H - H;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < sl; i += (long long)gridDim.x * blockDim.x) {
+        const long long n = first + i;
+        dst[i] = n < 0 ? 0.f : w[i] * ring[c * R + n % R];
+    }
+}
+
+// Overlap-add of reconstructed slices s0 .. s1 into the output ring, older slice first:
+// block b = [bH, (b+1)H) = second half of slice b (or what the ring already holds when b < s0)
+//                         + first half of slice b + 1 (when b + 1 <= s1).
+__global__ void slicq_ola_kernel(const float *stage, float *ring, long long R, long long sl, long long H, long long s0,
+                                 long long s1, int C) {
+    const int c = blockIdx.y;
+    const long long lo = (s0 - 1) * H, hi = (s1 + 1) * H;
+    for (long long n = lo + blockIdx.x * (long long)blockDim.x + threadIdx.x; n < hi; n += (long long)gridDim.x * blockDim.x) {
+        if (n < 0) continue;
+        const long long b = n / H, r = n - b * H;
+        float v = b >= s0 ? stage[((b - s0) * C + c) * sl + H + r] : ring[c * R + n % R];
+        if (b + 1 <= s1) v += stage[((b + 1 - s0) * C + c) * sl + r];
+        ring[c * R + n % R] = v;
+    }
+}
+
+__global__ void slicq_emit_kernel(const float *ring, long long R, long long pos, float *y, long long y_stride, long long n) {
+    const int c = blockIdx.y;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        y[c * y_stride + i] = ring[c * R + (pos + i) % R];
+}
+
+unsigned blocks_for(long long n) { return (unsigned)std::min<long long>(1024, std::max<long long>(1, (n + 255) / 256)); }
+
+cqt_status analyse_ready(cqt_slicq *s, cudaStream_t st) {
+    const int64_t ready = s->n_in / s->H;   // slices 0 .. ready - 1 are complete: (s + 1) H <= n_in
+    while (s->next_slice < ready) {
+        // slices whose coefficient slots are consecutive in memory
+        const int64_t slot = s->next_slice % s->K;
+        const int64_t cnt = std::min<int64_t>(ready - s->next_slice, s->K - slot);
+        dim3 grid(blocks_for(s->sl), (unsigned)(cnt * s->C));
+        slicq_cut_kernel<<<grid, 256, 0, st>>>(s->d_in, s->ring_in, s->d_win, s->d_stage, s->sl, s->H, s->next_slice, s->C);
+        if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+        cqt_status r = cqt_analyse(s->plan, s->d_stage, s->sl, cnt * s->C, s->sl,
+                                   s->d_coef + slot * s->C * cqt_plan_coeff_count(s->plan), s->d_ws, s->ws_bytes, st);
+        if (r != CQT_OK) return r;
+        s->next_slice += cnt;
+    }
+    return CQT_OK;
+}
+
+cqt_status push_impl(cqt_slicq *s, const float *x, int64_t x_stride, int64_t n, int zero, cudaStream_t st) {
+    // slices this push completes must fit the free coefficient slots
+    const int64_t will_be_ready = (s->n_in + n) / s->H;
+    if (will_be_ready - s->next_synth > s->K) return CQT_ERR_STATE;
+    int64_t done = 0;
+    while (done < n) {
+        // the ring must keep every sample from (next_slice - 1) H on
+        const int64_t oldest = std::max<int64_t>(0, (s->next_slice - 1) * s->H);
+        const int64_t room = s->ring_in - (s->n_in - oldest);
+        const int64_t m = std::min<int64_t>(n - done, room);
+        if (m <= 0) return CQT_ERR_STATE;
+        dim3 grid(blocks_for(m), (unsigned)s->C);
+        slicq_ingest_kernel<<<grid, 256, 0, st>>>(zero ? nullptr : x + done, x_stride, s->d_in, s->ring_in, s->n_in, m, zero);
+        if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+        s->n_in += m;
+        done += m;
+        cqt_status r = analyse_ready(s, st);
+        if (r != CQT_OK) return r;
+    }
+    return CQT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+cqt_status slicq_create(const cqt_plan *plan, int channels, int64_t transition, int64_t max_slices_in_flight,
+                        cqt_slicq **out) {
+    if (!plan || !out || channels < 1 || max_slices_in_flight < 1) return CQT_ERR_INVALID_ARG;
+    if (plan->device < 0) return CQT_ERR_STATE;
+    const int64_t sl = plan->N, H = sl / 2;
+    if (transition <= 0 || transition > H) return CQT_ERR_INVALID_ARG;
+    if (max_slices_in_flight * channels > 65535) return CQT_ERR_INVALID_ARG;
+    cqt_slicq *s = new (std::nothrow) cqt_slicq();
+    if (!s) return CQT_ERR_CUDA;
+    s->plan = plan; s->C = channels; s->sl = sl; s->H = H; s->tr = transition; s->K = max_slices_in_flight;
+    s->ring_in = (s->K + 2) * H;
+    s->ring_out = (s->K + 2) * H;
+    // Tukey slice window: 1 in the middle, raised-cosine flanks of `transition` samples centred on +-H/2
+    std::vector<float> w(sl);
+    const double lo = (H - transition) / 2.0, hi = (H + transition) / 2.0;
+    for (int64_t i = 0; i < sl; ++i) {
+        const double t = std::fabs((double)(i - sl / 2));
+        double v = 0.0;
+        if (t <= lo) v = 1.0;
+        else if (t < hi) v = 0.5 * (1.0 + std::cos(3.14159265358979323846 * (t - lo) / (double)transition));
+        w[i] = (float)v;
+    }
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cudaSetDevice(plan->device) != cudaSuccess) { delete s; return CQT_ERR_CUDA; }
+    const int64_t cc = cqt_plan_coeff_count(plan);
+    s->ws_bytes = cqt_plan_workspace_bytes(plan, s->K * channels);
+    const size_t b_win = sl * sizeof(float), b_in = (size_t)channels * s->ring_in * sizeof(float),
+                 b_stage = (size_t)s->K * channels * sl * sizeof(float), b_coef = (size_t)s->K * channels * cc * sizeof(cqt_c64),
+                 b_out = (size_t)channels * s->ring_out * sizeof(float);
+    cudaError_t e = cudaSuccess;
+    auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+    chk(cudaMalloc((void **)&s->d_win, b_win));
+    chk(cudaMalloc((void **)&s->d_in, b_in));
+    chk(cudaMalloc((void **)&s->d_stage, b_stage));
+    chk(cudaMalloc((void **)&s->d_coef, b_coef));
+    chk(cudaMalloc((void **)&s->d_out, b_out));
+    chk(cudaMalloc(&s->d_ws, s->ws_bytes));
+    if (e == cudaSuccess) chk(cudaMemcpy(s->d_win, w.data(), b_win, cudaMemcpyHostToDevice));
+    if (e == cudaSuccess) chk(cudaMemset(s->d_out, 0, b_out));
+    s->total_bytes = b_win + b_in + b_stage + b_coef + b_out + s->ws_bytes;
+    cudaSetDevice(cur);
+    if (e != cudaSuccess) { slicq_destroy(s); return CQT_ERR_CUDA; }
+    *out = s;
+    return CQT_OK;
+}
+
+cqt_status slicq_push(cqt_slicq *s, const float *x, int64_t x_stride, int64_t n, void *stream, int64_t *slices_completed) {
+    if (!s || n < 0 || (n > 0 && (!x || x_stride < n))) return CQT_ERR_INVALID_ARG;
+    cqt_status r = n > 0 ? push_impl(s, x, x_stride, n, 0, reinterpret_cast<cudaStream_t>(stream)) : CQT_OK;
+    if (slices_completed) *slices_completed = s->next_slice;
+    return r;
+}
+
+cqt_status slicq_flush(cqt_slicq *s, void *stream) {
+    if (!s) return CQT_ERR_INVALID_ARG;
+    // enough zeros that every frame pushed so far becomes final: n_in -> (ceil(n_in / H) + 1) H
+    const int64_t target = ((s->n_in + s->H - 1) / s->H + 1) * s->H;
+    return push_impl(s, nullptr, 0, target - s->n_in, 1, reinterpret_cast<cudaStream_t>(stream));
+}
+
+cqt_status slicq_coeffs(cqt_slicq *s, int64_t slice_index, cqt_c64 **c) {
+    if (!s || !c) return CQT_ERR_INVALID_ARG;
+    if (slice_index < s->next_synth || slice_index >= s->next_slice) return CQT_ERR_STATE;
+    *c = s->d_coef + (slice_index % s->K) * s->C * cqt_plan_coeff_count(s->plan);
+    return CQT_OK;
+}
+
+cqt_status slicq_pull(cqt_slicq *s, float *y, int64_t y_stride, int64_t n_max, void *stream, int64_t *n_written) {
+    if (!s || n_max < 0 || (n_max > 0 && (!y || y_stride < n_max)) || !n_written) return CQT_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int64_t written = 0;
+    for (;;) {
+        // synthesise as many pending slices as the output ring has room for
+        while (s->next_synth < s->next_slice) {
+            // the ring holds frames n_out .. next_synth * H - 1; every slice adds H frames
+            const int64_t room_slices = (s->ring_out - (s->next_synth * s->H - s->n_out)) / s->H;
+            const int64_t slot = s->next_synth % s->K;
+            const int64_t cnt = std::min<int64_t>({s->next_slice - s->next_synth, s->K - slot, room_slices});
+            if (cnt <= 0) break;
+            cqt_status r = cqt_synthesise(s->plan, s->d_coef + slot * s->C * cqt_plan_coeff_count(s->plan), cnt * s->C, s->sl,
+                                          s->d_stage, s->sl, s->d_ws, s->ws_bytes, st);
+            if (r != CQT_OK) return r;
+            dim3 grid(blocks_for((cnt + 1) * s->H), (unsigned)s->C);
+            slicq_ola_kernel<<<grid, 256, 0, st>>>(s->d_stage, s->d_out, s->ring_out, s->sl, s->H, s->next_synth,
+                                                   s->next_synth + cnt - 1, s->C);
+            if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+            s->next_synth += cnt;
+        }
+        // frames below (next_synth - 1) H are final
+        const int64_t final_to = std::max<int64_t>(0, (s->next_synth - 1) * s->H);
+        const int64_t m = std::min<int64_t>(n_max - written, final_to - s->n_out);
+        if (m > 0) {
+            dim3 grid(blocks_for(m), (unsigned)s->C);
+            slicq_emit_kernel<<<grid, 256, 0, st>>>(s->d_out, s->ring_out, s->n_out, y + written, y_stride, m);
+            if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+            s->n_out += m;
+            written += m;
+        }
+        if (m <= 0 || written >= n_max || s->next_synth >= s->next_slice) break;
+    }
+    *n_written = written;
+    return CQT_OK;
+}
+
+cqt_status slicq_reset(cqt_slicq *s) {
+    if (!s) return CQT_ERR_INVALID_ARG;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    cudaSetDevice(s->plan->device);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemset(s->d_out, 0, (size_t)s->C * s->ring_out * sizeof(float));
+    cudaSetDevice(cur);
+    s->n_in = s->next_slice = s->next_synth = s->n_out = 0;
+    return e == cudaSuccess ? CQT_OK : CQT_ERR_CUDA;
+}
+
+cqt_status slicq_destroy(cqt_slicq *s) {
+    if (!s) return CQT_OK;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    cudaSetDevice(s->plan->device);
+    cudaFree(s->d_win); cudaFree(s->d_in); cudaFree(s->d_stage); cudaFree(s->d_coef); cudaFree(s->d_out); cudaFree(s->d_ws);
+    cudaSetDevice(cur);
+    delete s;
+    return CQT_OK;
+}
+
+size_t slicq_device_bytes(const cqt_slicq *s) { return s ? s->total_bytes : 0; }
+
+}  // extern "C"

@@ -1,0 +1,147 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded inputs.
+
+Tolerances (fp32 arithmetic against an fp64 reference): per band ||c_gpu - c_oracle||_2 / ||c_oracle||_2 <= 1e-5;
+signals from synthesis / adjoints <= 1e-5 relative L2; round trip SNR >= 120 dB on the true samples."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from helpers import band_rel_errors, library_plan, oracle_layout, small_workload, snr_db, split_bands
+from oracle import nsgt_oracle as orc
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+CASES = [
+    small_workload("n256"),
+    small_workload("n256_bh_smooth", window=wl.WIN_BLACKMAN_HARRIS, m_policy=wl.M_SMOOTH),
+    small_workload("n4096_b48", N=4096, valid_len=4096, fs=22050.0, fmin=200.0, fmax=11025.0, bins_per_octave=48,
+                   m_policy=wl.M_SMOOTH, channels=3),
+    small_workload("n4096_ragged", N=4096, valid_len=3001, fs=22050.0, fmin=200.0, fmax=11025.0, bins_per_octave=12,
+                   m_policy=wl.M_MULT4, channels=3),
+    small_workload("n16384_mult4", N=1 << 14, valid_len=1 << 14, fs=44100.0, fmin=32.70, fmax=22050.0,
+                   bins_per_octave=12, m_policy=wl.M_MULT4, channels=2),
+    small_workload("slice_2e15", N=1 << 15, valid_len=1 << 15, fs=44100.0, fmin=32.70, fmax=22050.0,
+                   bins_per_octave=48, m_policy=wl.M_SMOOTH, channels=2),
+    wl.CONFIGS["config1"],
+    small_workload("n65536_ragged_pow2", N=1 << 16, valid_len=50001, fs=44100.0, fmin=32.70, fmax=22050.0,
+                   bins_per_octave=12, m_policy=wl.M_POW2, channels=3),
+    wl.scaled(wl.CONFIGS["config3"], channels=2),
+]
+
+
+@pytest.fixture(scope="module", params=CASES, ids=lambda w: w.name)
+def case(request):
+    w = request.param
+    lay = oracle_layout(w)
+    plan = library_plan(w)
+    x = wl.make_signal(w)
+    yield w, lay, plan, x
+    plan.close()
+
+
+def test_analysis_matches_oracle_per_band(case):
+    w, lay, plan, x = case
+    c = plan.analyse(_dev(x), valid_len=w.valid_len).cpu().numpy()
+    want = orc.analyse(lay, orc.pad_signal(x, w.N))
+    errs = band_rel_errors(lay, c, want)
+    assert errs.max() <= TOL, (int(errs.argmax()), errs.max())
+
+
+def test_synthesis_matches_oracle_on_arbitrary_coefficients(case):
+    w, lay, plan, x = case
+    y = wl.make_cotangent(w, lay.coeff_count)
+    got = plan.synthesise(_dev(y), valid_len=w.valid_len).cpu().numpy()
+    want = orc.synthesise(lay, split_bands(lay, y.astype(np.complex128)))[..., :w.valid_len]
+    rel = np.linalg.norm(got - want, axis=-1) / np.linalg.norm(want, axis=-1)
+    assert rel.max() <= TOL, rel
+
+
+def test_round_trip_snr(case):
+    w, lay, plan, x = case
+    xd = _dev(x)
+    c = plan.analyse(xd, valid_len=w.valid_len)
+    xr = plan.synthesise(c, valid_len=w.valid_len).cpu().numpy()
+    if w.valid_len == w.N:
+        assert snr_db(x, xr).min() >= 120.0, snr_db(x, xr)
+    else:
+        # truncating the reconstruction of a zero-padded signal: compare on the true samples
+        assert snr_db(x, xr).min() >= 120.0, snr_db(x, xr)
+
+
+def test_adjoints_match_oracle(case):
+    w, lay, plan, x = case
+    y = wl.make_cotangent(w, lay.coeff_count)
+    got = plan.analyse_adjoint(_dev(y), valid_len=w.valid_len).cpu().numpy()
+    want = orc.analyse_adjoint(lay, split_bands(lay, y.astype(np.complex128)))[..., :w.valid_len]
+    rel = np.linalg.norm(got - want, axis=-1) / np.linalg.norm(want, axis=-1)
+    assert rel.max() <= TOL, rel
+    cb = plan.synthesise_adjoint(_dev(x), valid_len=w.valid_len).cpu().numpy()
+    want_c = orc.synthesise_adjoint(lay, orc.pad_signal(x, w.N))
+    errs = band_rel_errors(lay, cb, want_c)
+    assert errs.max() <= TOL, (int(errs.argmax()), errs.max())
+
+
+def test_adjoint_identity_on_gpu_outputs(case):
+    """<T x, y> = <x, T' y> and <S y, xb> = <y, S' xb> with every operand computed by the kernels."""
+    w, lay, plan, x = case
+    y = wl.make_cotangent(w, lay.coeff_count)
+    xd, yd = _dev(x), _dev(y)
+    Tx = plan.analyse(xd, valid_len=w.valid_len).cpu().numpy().astype(np.complex128)
+    Tty = plan.analyse_adjoint(yd, valid_len=w.valid_len).cpu().numpy().astype(np.float64)
+    Sy = plan.synthesise(yd, valid_len=w.valid_len).cpu().numpy().astype(np.float64)
+    Stx = plan.synthesise_adjoint(xd, valid_len=w.valid_len).cpu().numpy().astype(np.complex128)
+    y64, x64 = y.astype(np.complex128), x.astype(np.float64)
+    for ch in range(x.shape[0]):
+        lhs, rhs = np.real(np.vdot(Tx[ch], y64[ch])), np.dot(x64[ch], Tty[ch])
+        assert abs(lhs - rhs) <= 2e-5 * np.linalg.norm(Tx[ch]) * np.linalg.norm(y64[ch])
+        lhs, rhs = np.dot(Sy[ch], x64[ch]), np.real(np.vdot(y64[ch], Stx[ch]))
+        assert abs(lhs - rhs) <= 2e-5 * np.linalg.norm(Sy[ch]) * np.linalg.norm(x64[ch])
+
+
+def test_bitwise_reproducible(case):
+    w, lay, plan, x = case
+    xd = _dev(x)
+    c1 = plan.analyse(xd, valid_len=w.valid_len)
+    c2 = plan.analyse(xd, valid_len=w.valid_len)
+    assert torch.equal(torch.view_as_real(c1), torch.view_as_real(c2))
+    x1 = plan.synthesise(c1, valid_len=w.valid_len)
+    x2 = plan.synthesise(c1, valid_len=w.valid_len)
+    assert torch.equal(x1, x2)
+
+
+def test_row_stride_and_padding_are_respected():
+    w = CASES[3]
+    plan = library_plan(w)
+    x = wl.make_signal(w)
+    wide = torch.full((w.channels, w.valid_len + 37), 7.0, device="cuda")
+    wide[:, :w.valid_len] = _dev(x)
+    c_wide = plan.analyse(wide, valid_len=w.valid_len)
+    c_ref = plan.analyse(_dev(x), valid_len=w.valid_len)
+    assert torch.equal(torch.view_as_real(c_wide), torch.view_as_real(c_ref))
+    out = torch.full((w.channels, w.valid_len + 5), -3.0, device="cuda")
+    plan.synthesise(c_ref, valid_len=w.valid_len, out=out)
+    assert torch.all(out[:, w.valid_len:] == -3.0)          # nothing written past valid_len
+    plan.close()
+
+
+def test_argument_errors_on_device_plan():
+    from paper_2609_29119_b200 import CqtError
+    w = CASES[0]
+    plan = library_plan(w)
+    x = _dev(wl.make_signal(w))
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(CqtError) as e:
+        plan.analyse(x, ws=small)
+    assert e.value.status == -4
+    with pytest.raises(CqtError) as e:
+        plan.analyse(x, valid_len=w.N + 2)
+    assert e.value.status == -1
+    plan.close()
