@@ -1,0 +1,339 @@
+#!/usr/bin/env python3
+"""Benchmark of the constant-Q analysis + synthesis round trip on B200.
+
+A step is one pass of the whole hot path over one batch: cqt_analyse then cqt_synthesise of
+every signal of the workload (default: 16 stereo clips of 10 s at 44.1 kHz, N = 2^19, 24 bins
+per octave).  Prints one JSON line ("Measurement").
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload configN]
+
+--impl reference times the fp64 CPU oracle (the only reference implementation that exists for
+this method) on a bounded sample of the same workload on the host cores.
+With N > 1 ranks every rank runs an independent replica of the batch (the transform has no
+exchange step); `value` is the job's aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads as wl  # noqa: E402
+
+METRIC = "cqt_round_trip_throughput"
+UNIT = "Msamples/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(w: wl.Workload, budget_macs: float = 1.2e8):
+    """Times the oracle on ONE channel of the workload, all of the long DFT and a strided subset of the bands
+    (analysis and synthesis by direct per-band DFT), and extrapolates by the share of direct-DFT work sampled."""
+    from threadpoolctl import threadpool_limits
+
+    from oracle import nsgt_oracle as orc
+    lay = orc.build_layout(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, policy=w.m_policy,
+                           min_win=w.min_win)
+    x = orc.pad_signal(wl.make_signal(w, n_channels=1)[0].astype(np.float64), w.N)
+    work = np.array([float(b.M) * len(b.d) for b in lay.bands])
+    # every stride-th band, smallest stride that keeps the sampled work under the budget
+    stride = 1
+    while work[::stride].sum() > budget_macs and stride < len(lay.bands):
+        stride += 1
+    sel = list(range(0, len(lay.bands), stride))
+    frac = float(work[sel].sum() / work.sum())
+    with threadpool_limits(limits=1):
+        t0 = time.perf_counter()
+        X = orc.long_dft(x)
+        t1 = time.perf_counter()
+        c = [orc.analyse_band(lay, X, i) for i in sel]
+        t2 = time.perf_counter()
+        orc.synthesise(lay, c, bands=sel)      # includes the inverse long DFT
+        t3 = time.perf_counter()
+    # long DFTs are done in full; the band work is scaled up to all bands
+    t_long = (t1 - t0) * 2.0
+    t_band_an = (t2 - t1) / frac
+    t_band_sy = max(0.0, (t3 - t2) - (t1 - t0)) / frac
+    est = t_long + t_band_an + t_band_sy
+    return {"seconds_measured": t3 - t0, "seconds_full_round_trip_one_channel": est,
+            "msamples_per_s": w.valid_len / est / 1e6, "work_fraction": frac, "bands_sampled": len(sel),
+            "bands": len(lay.bands)}
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals, last = [], None
+    for i in range(args.warmup + args.steps):
+        last = oracle_sample(w, budget_macs=args.cpu_budget_macs)
+        if i >= args.warmup:
+            vals.append(last)
+    est = statistics.mean(v["seconds_full_round_trip_one_channel"] for v in vals)
+    value = w.valid_len / est / 1e6
+    sample = (f"1 of {w.channels} channels; both long DFTs in full; {last['bands_sampled']} of {last['bands']} bands "
+              f"({100 * last['work_fraction']:.2f} % of the direct-DFT work) analysed and synthesised, "
+              f"band time scaled to all bands")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": est * w.channels * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "channels": w.channels, "valid_len": w.valid_len, "N": w.N,
+                       "bins_per_octave": w.bins_per_octave},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU arm
+class ClockSampler:
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+                 "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+                 "clocks_event_reasons.sw_power_cap")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "50",
+                                          "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                p = [v.strip() for v in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0])); mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def kernel_algorithmic_bytes(plan, w, batch):
+    """Minimal HBM bytes each kernel is responsible for per launch: signal samples, coefficients and window
+    tables; the packed spectrum, the half spectrum and the weighted-bin rows are intermediates (0 bytes)."""
+    cls_m = {}
+    cls_s = {}
+    for bi in plan.bands():
+        cls_m[bi.launch_class] = cls_m.get(bi.launch_class, 0) + bi.M
+        cls_s[bi.launch_class] = cls_s.get(bi.launch_class, 0) + bi.support
+    sig = 4 * w.valid_len * batch
+    two_pass = plan.N // 2 > 16384
+    out = {"rfft_cols_fwd": sig if two_pass else 0, "rfft_rows_fwd": 0 if two_pass else sig,
+           "irfft_cols": sig if two_pass else 0, "irfft_rows": 0 if two_pass else sig}
+    for c in cls_m:
+        b = 8 * cls_m[c] * batch + 4 * cls_s[c]
+        out[f"bands_from_spectrum/class{c}"] = b
+        out[f"bands_to_spectrum/class{c}"] = b
+    return out
+
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_29119_b200 import Plan
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    dev = torch.device(f"cuda:{local}")
+    batch = w.channels
+    plan = Plan(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, m_policy=w.m_policy, min_win=w.min_win,
+                device=local)
+    x_host = torch.from_numpy(wl.make_signal(w)).pin_memory()
+    xr_host = torch.empty_like(x_host).pin_memory()
+    x = x_host.to(dev)
+    c = torch.empty((batch, plan.coeff_count), dtype=torch.complex64, device=dev)
+    xr = torch.empty_like(x)
+    ws = plan.workspace(batch)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        plan.analyse(x, valid_len=w.valid_len, out=c, ws=ws, stream=stream)
+        plan.synthesise(c, valid_len=w.valid_len, out=xr, ws=ws, stream=stream)
+
+    def step_e2e():
+        x.copy_(x_host, non_blocking=True)
+        step()
+        xr_host.copy_(xr, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, k):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(k):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    W, K = max(3, args.warmup), args.steps
+    for _ in range(W):
+        step()
+    torch.cuda.synchronize()
+    # correctness guard of the timed configuration: fp32 round trip >= 120 dB on every channel
+    xd, xrd = x.double(), xr.double()
+    snr = 10 * torch.log10((xd * xd).sum(1) / ((xd - xrd) ** 2).sum(1))
+    snr_min = float(snr.min().item())
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = plan.launch_count()
+    ms = timed(step, K)
+    launches = plan.launch_count() - launches0
+    clocks = sampler.stop()
+
+    # per-kernel durations: the same K steps with an event after every kernel
+    plan.set_timing(True)
+    for _ in range(K):
+        step()
+    per = {}
+    for name, t in plan.read_timing(capacity=64 * K + 64):
+        a = per.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += t
+    plan.set_timing(False)
+
+    for _ in range(2):
+        step_e2e()
+    ms_e2e = timed(step_e2e, K)
+
+    samples = float(batch) * w.valid_len * world
+    value = samples / (ms / K / 1e3) / 1e6
+    e2e_value = samples / (ms_e2e / K / 1e3) / 1e6
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    alg = kernel_algorithmic_bytes(plan, w, batch)
+    tot_ms = sum(v[1] for v in per.values())
+    kernels = {n: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0], "share": v[1] / tot_ms,
+                   "alg_bytes": alg.get(n, 0),
+                   "alg_gbs": alg.get(n, 0) / (v[1] / v[0] * 1e-3) / 1e9} for n, v in per.items()}
+    dom = max(per, key=lambda n: per[n][1])
+    dom_gbs = kernels[dom]["alg_gbs"]
+    path_bytes = sum(alg.values())
+    path_gbs = path_bytes / (ms / K * 1e-3) / 1e9
+    traffic = None
+    prof = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(prof):
+        try:
+            traffic = json.load(open(prof)).get(w.name, {}).get(dom)
+        except Exception:
+            traffic = None
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        s = oracle_sample(w, budget_macs=args.cpu_budget_macs)
+        cpu = {"value": s["msamples_per_s"], "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": (f"1 of {w.channels} channels; both long DFTs in full; {s['bands_sampled']} of {s['bands']} bands "
+                          f"({100 * s['work_fraction']:.2f} % of the direct-DFT work), band time scaled to all bands; "
+                          f"{s['seconds_measured']:.1f} s measured")}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "channels_per_gpu": batch, "valid_len": w.valid_len, "N": w.N,
+                   "bins_per_octave": w.bins_per_octave, "bands": plan.num_bands, "coeffs_per_channel": plan.coeff_count,
+                   "round_trips_per_s": batch * world / (ms / K / 1e3), "l2": "inputs larger than L2 (no flush)",
+                   "multi_gpu": "replicas only", "round_trip_snr_db_min": snr_min},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
+                "d2h_bytes_per_step": int(xr_host.numel() * 4), "ms_per_step": ms_e2e / K},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": dom_gbs / peak, "traffic": traffic, "peak_kind": peak_kind,
+                     "path_achieved": path_gbs, "path_frac": path_gbs / peak, "path_alg_bytes": path_bytes},
+        "kernels": kernels,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--channels", type=int, default=None, help="override the number of signals (profiling on small cases)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget-macs", type=float, default=1.2e8)
+    args = ap.parse_args()
+    w = wl.CONFIGS[args.workload]
+    if args.channels:
+        w = wl.scaled(w, channels=args.channels)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

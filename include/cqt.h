@@ -83,6 +83,7 @@ typedef struct {
     int64_t coeff_offset; /* into one signal's coefficient row */
     int64_t table_offset; /* into the g / h tables returned by cqt_plan_tables */
     int is_sideband;      /* 0 regular, 1 DC, 2 Nyquist */
+    int launch_class;     /* which of the band kernels' length classes (0 = shortest) runs this band */
 } cqt_band_info;
 
 typedef struct cqt_plan cqt_plan;
@@ -115,6 +116,18 @@ size_t cqt_plan_workspace_bytes(const cqt_plan *plan, int64_t batch);
 cqt_status cqt_plan_tables(const cqt_plan *plan, const float **g_host, const float **h_host);
 /* Reserved for device-side self checks; returns CQT_OK in release builds. May synchronise. */
 cqt_status cqt_plan_check(const cqt_plan *plan);
+
+/*
+ * Benchmark aids (the paper has no counterpart).  cqt_plan_launch_count: kernels launched through this
+ * plan since it was created.  cqt_plan_set_timing(plan, 1): every later transform call records a CUDA
+ * event on its stream before its first kernel and after each kernel; cqt_plan_read_timing waits for those
+ * events, returns for each kernel launched since the last read its name (static strings) and its
+ * duration in milliseconds (at most `capacity` entries are written; *count receives the total), and clears
+ * the record.  Not thread safe; leave timing off in production calls.
+ */
+int64_t cqt_plan_launch_count(const cqt_plan *plan);
+cqt_status cqt_plan_set_timing(const cqt_plan *plan, int enable);
+cqt_status cqt_plan_read_timing(const cqt_plan *plan, const char **names, float *ms, int64_t capacity, int64_t *count);
 
 /*
  * Analysis T (Eq. analysis, band-spectrum, packed-analysis):
@@ -173,7 +186,9 @@ cqt_status cqt_synthesise_adjoint(const cqt_plan *plan, const float *x_bar, int6
  *                first) and writes up to n_max finished frames per channel to y (device,
  *                [channels][n_max], row stride y_stride); *n_written (host) receives the count.  Frame n
  *                is finished once slice floor(n / (sl/2)) + 1 has been synthesised: one slice of latency.
- *   slicq_flush  pushes sl/2 zeros per channel so the tail of the stream can be pulled.
+ *   slicq_flush  pushes zeros (between sl/2 and sl per channel) up to the next multiple of sl/2 plus sl/2, so
+ *                that every frame pushed so far becomes final and can be pulled.
+ *   Push, pull and flush of one object must be issued on the same stream (they share staging buffers).
  *   slicq_reset  drops all state and restarts at slice 0 (synchronises the object's stream use).
  */
 cqt_status slicq_create(const cqt_plan *slice_plan, int channels, int64_t transition,

@@ -290,11 +290,12 @@ def analyse_band(lay: Layout, X: np.ndarray, band: int, n: Optional[np.ndarray] 
     return _direct_band_sum(vals, b.d, np.asarray(n, dtype=np.int64), b.M, +1) / b.M
 
 
-def analyse(lay: Layout, x: np.ndarray) -> List[np.ndarray]:
-    """T x: list over bands of arrays [..., M_lambda]."""
+def analyse(lay: Layout, x: np.ndarray, bands: Optional[Sequence[int]] = None) -> List[np.ndarray]:
+    """T x: list over bands (all, or the listed ones) of arrays [..., M_lambda]."""
     x = np.asarray(x, dtype=np.float64)
     X = long_dft(x)
-    return [analyse_band(lay, X, i) for i in range(len(lay.bands))]
+    idx = range(len(lay.bands)) if bands is None else bands
+    return [analyse_band(lay, X, i) for i in idx]
 
 
 def pad_signal(x: np.ndarray, N: int) -> np.ndarray:
@@ -310,11 +311,13 @@ def pad_signal(x: np.ndarray, N: int) -> np.ndarray:
 # synthesis  x^ = F_N^{-1} sum_lambda diag(h_lambda) E_lambda^T F_M c_lambda   (Eq. synthesis)
 # --------------------------------------------------------------------------
 
-def synthesise(lay: Layout, c: Sequence[np.ndarray]) -> np.ndarray:
+def synthesise(lay: Layout, c: Sequence[np.ndarray], bands: Optional[Sequence[int]] = None) -> np.ndarray:
+    """S c.  With `bands`, c lists only those bands and the others contribute nothing."""
     N = lay.N
     lead = np.asarray(c[0]).shape[:-1]
     Xh = np.zeros(lead + (N // 2 + 1,), dtype=np.complex128)
-    for b, cb in zip(lay.bands, c):
+    which = lay.bands if bands is None else [lay.bands[i] for i in bands]
+    for b, cb in zip(which, c):
         cb = np.asarray(cb, dtype=np.complex128)
         k = b.kc + b.d
         ok = (k >= 0) & (k <= N // 2)

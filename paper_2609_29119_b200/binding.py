@@ -32,7 +32,7 @@ class PlanDesc(C.Structure):
 class BandInfo(C.Structure):
     _fields_ = [("centre_hz", C.c_double), ("centre_bin", C.c_int64), ("support", C.c_int64),
                 ("first_offset", C.c_int64), ("M", C.c_int64), ("coeff_offset", C.c_int64),
-                ("table_offset", C.c_int64), ("is_sideband", C.c_int)]
+                ("table_offset", C.c_int64), ("is_sideband", C.c_int), ("launch_class", C.c_int)]
 
 
 EXPORTS = {
@@ -47,6 +47,9 @@ EXPORTS = {
     "cqt_plan_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int64]),
     "cqt_plan_tables": (C.c_int, [C.c_void_p, C.POINTER(C.POINTER(C.c_float)), C.POINTER(C.POINTER(C.c_float))]),
     "cqt_plan_check": (C.c_int, [C.c_void_p]),
+    "cqt_plan_launch_count": (C.c_int64, [C.c_void_p]),
+    "cqt_plan_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
+    "cqt_plan_read_timing": (C.c_int, [C.c_void_p, C.POINTER(C.c_char_p), C.POINTER(C.c_float), C.c_int64, C.POINTER(C.c_int64)]),
     "cqt_analyse": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "cqt_synthesise": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]),
     "cqt_analyse_adjoint": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -156,6 +159,21 @@ class Plan:
             self._ws = torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}")
         return self._ws
 
+    def launch_count(self) -> int:
+        return int(self.lib.cqt_plan_launch_count(self.handle))
+
+    def set_timing(self, enable: bool) -> None:
+        _check(self.lib.cqt_plan_set_timing(self.handle, 1 if enable else 0), "cqt_plan_set_timing")
+
+    def read_timing(self, capacity: int = 4096):
+        """[(kernel name, milliseconds)] for every kernel launched since the last read (synchronises)."""
+        names = (C.c_char_p * capacity)()
+        ms = (C.c_float * capacity)()
+        n = C.c_int64()
+        _check(self.lib.cqt_plan_read_timing(self.handle, names, ms, capacity, C.byref(n)), "cqt_plan_read_timing")
+        m = min(int(n.value), capacity)
+        return [(names[i].decode(), float(ms[i])) for i in range(m)]
+
     # ---- transforms (x: [batch, >= valid_len] float32 cuda; c: [batch, coeff_count] complex64 cuda)
     def _sig(self, x, valid_len):
         import torch
@@ -242,15 +260,15 @@ class SliCQ:
         _check(self.lib.slicq_reset(self.handle), "slicq_reset")
 
 
+class _DeviceArray:
+    """Exposes a device buffer owned by the library through the CUDA array interface."""
+
+    def __init__(self, ptr: int, shape):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": "<c8", "data": (ptr, False), "version": 3,
+                                         "strides": None}
+
+
 def _DevicePtrTensor(ptr: int, shape, device: int):
-    """Copy of a device buffer owned by the library into a new complex64 torch tensor."""
+    """Zero-copy complex64 torch view of a device buffer owned by the library."""
     import torch
-    n = 1
-    for s in shape:
-        n *= s
-    out = torch.empty(shape, dtype=torch.complex64, device=f"cuda:{device}")
-    cudart = torch.cuda.cudart()
-    err = cudart.cudaMemcpy(out.data_ptr(), ptr, n * 8, 3)  # cudaMemcpyDeviceToDevice
-    if int(err) != 0:
-        raise RuntimeError(f"cudaMemcpy failed: {err}")
-    return out
+    return torch.as_tensor(_DeviceArray(ptr, shape), device=f"cuda:{device}")

@@ -110,6 +110,7 @@ void free_device(cqt_plan *p) {
     cudaFree(p->d.tab_analysis_adj); cudaFree(p->d.tab_synthesis_adj);
     cudaFree(p->d.cover); cudaFree(p->d.span);
     for (auto &c : p->cls) cudaFree(c.d_work);
+    for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     cudaSetDevice(cur);
 }
 
@@ -289,6 +290,10 @@ cqt_status cqt_plan_band_info(const cqt_plan *p, int64_t band, cqt_band_info *ou
     const HostBand &hb = p->lay.bands[band];
     out->centre_hz = hb.centre_hz; out->centre_bin = hb.kc; out->support = hb.S; out->first_offset = hb.d0;
     out->M = hb.M; out->coeff_offset = hb.coeff_off; out->table_offset = hb.tab_off; out->is_sideband = hb.side;
+    out->launch_class = 0;
+    for (int c = 0; c < kNumClasses; ++c)
+        for (int32_t b : p->cls[c].work)
+            if (b == band) out->launch_class = c;
     return CQT_OK;
 }
 
@@ -307,6 +312,54 @@ cqt_status cqt_plan_tables(const cqt_plan *p, const float **g_host, const float 
 }
 
 cqt_status cqt_plan_check(const cqt_plan *p) { return p ? CQT_OK : CQT_ERR_INVALID_ARG; }
+
+}  // extern "C"
+
+namespace cqt {
+
+void note_launch(const cqt_plan &p, const char *name, cudaStream_t st) {
+    if (name) ++p.launches;
+    if (!p.timing) return;
+    if (p.ev_used == p.ev.size()) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        p.ev.push_back(e);
+        p.ev_name.push_back(nullptr);
+    }
+    p.ev_name[p.ev_used] = name;
+    cudaEventRecord(p.ev[p.ev_used], st);
+    ++p.ev_used;
+}
+
+}  // namespace cqt
+
+extern "C" {
+
+int64_t cqt_plan_launch_count(const cqt_plan *p) { return p ? p->launches : -1; }
+
+cqt_status cqt_plan_set_timing(const cqt_plan *p, int enable) {
+    if (!p) return CQT_ERR_INVALID_ARG;
+    p->timing = enable != 0;
+    p->ev_used = 0;
+    return CQT_OK;
+}
+
+cqt_status cqt_plan_read_timing(const cqt_plan *p, const char **names, float *ms, int64_t capacity, int64_t *count) {
+    if (!p || !count || capacity < 0 || (capacity > 0 && (!names || !ms))) return CQT_ERR_INVALID_ARG;
+    int64_t n = 0;
+    for (size_t i = 1; i < p->ev_used; ++i) {
+        if (!p->ev_name[i]) continue;   // start-of-call marker
+        if (n < capacity) {
+            if (cudaEventSynchronize(p->ev[i]) != cudaSuccess) return CQT_ERR_CUDA;
+            if (cudaEventElapsedTime(&ms[n], p->ev[i - 1], p->ev[i]) != cudaSuccess) return CQT_ERR_CUDA;
+            names[n] = p->ev_name[i];
+        }
+        ++n;
+    }
+    *count = n;
+    p->ev_used = 0;
+    return CQT_OK;
+}
 
 }  // extern "C"
 
@@ -332,6 +385,7 @@ cqt_status begin_call(const cqt_plan *p, const void *sig, int64_t stride, int64_
     c.st = reinterpret_cast<cudaStream_t>(stream);
     if (cudaGetDevice(&c.prev_dev) != cudaSuccess) return CQT_ERR_CUDA;
     if (c.prev_dev != p->device && cudaSetDevice(p->device) != cudaSuccess) return CQT_ERR_CUDA;
+    note_launch(*p, nullptr, c.st);
     return CQT_OK;
 }
 

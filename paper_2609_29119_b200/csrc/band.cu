@@ -136,7 +136,8 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
 }
 
 template <class K>
-static cudaError_t launch_class(K warp_kernel, K block_kernel, const BandClass &c, BandArgs &a, cudaStream_t st) {
+static cudaError_t launch_class(const cqt_plan &p, const char *name, K warp_kernel, K block_kernel, const BandClass &c,
+                                BandArgs &a, cudaStream_t st) {
     if (c.n_bands == 0) return cudaSuccess;
     const long long items = (long long)c.n_bands * a.batch;
     const size_t smem = (size_t)c.max_elems * c.items_per_cta * sizeof(float2);
@@ -145,6 +146,7 @@ static cudaError_t launch_class(K warp_kernel, K block_kernel, const BandClass &
         warp_kernel<<<(unsigned)grid, c.threads, smem, st>>>(a);
     else
         block_kernel<<<(unsigned)grid, c.threads, smem, st>>>(a);
+    note_launch(p, name, st);
     return cudaGetLastError();
 }
 
@@ -155,7 +157,9 @@ cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, co
         a.spec = X;
         a.spec_pitch = p.lf.x_pitch;
         a.coef = c;
-        cudaError_t e = launch_class(bands_from_spectrum_kernel<true>, bands_from_spectrum_kernel<false>, p.cls[i], a, st);
+        static const char *names[kNumClasses] = {"bands_from_spectrum/class0", "bands_from_spectrum/class1",
+                                                  "bands_from_spectrum/class2", "bands_from_spectrum/class3"};
+        cudaError_t e = launch_class(p, names[i], bands_from_spectrum_kernel<true>, bands_from_spectrum_kernel<false>, p.cls[i], a, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -168,7 +172,9 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
         a.coef = const_cast<float2 *>(c);
         a.Y = Y;
         a.fold = fold_sidebands ? 1 : 0;
-        cudaError_t e = launch_class(bands_to_spectrum_kernel<true>, bands_to_spectrum_kernel<false>, p.cls[i], a, st);
+        static const char *names[kNumClasses] = {"bands_to_spectrum/class0", "bands_to_spectrum/class1",
+                                                  "bands_to_spectrum/class2", "bands_to_spectrum/class3"};
+        cudaError_t e = launch_class(p, names[i], bands_to_spectrum_kernel<true>, bands_to_spectrum_kernel<false>, p.cls[i], a, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

@@ -60,12 +60,21 @@ struct cqt_plan {
     cqt::DevicePlan d;
     int max_smem_optin = 0;
     int sm_count = 0;
+    // launch counter and optional per-kernel event timing (benchmark aid; not thread safe)
+    mutable int64_t launches = 0;
+    mutable bool timing = false;
+    mutable std::vector<cudaEvent_t> ev;
+    mutable std::vector<const char *> ev_name;
+    mutable size_t ev_used = 0;
 };
 
 namespace cqt {
 
 // table selectors of the band kernels
 enum { TAB_ANALYSIS = 0, TAB_SYNTHESIS = 1, TAB_ANALYSIS_ADJ = 2, TAB_SYNTHESIS_ADJ = 3 };
+
+// api.cu: called after every kernel launch (and once at the start of a call with name == nullptr)
+void note_launch(const cqt_plan &p, const char *name, cudaStream_t st);
 
 // long_fft.cu
 cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,

@@ -292,6 +292,7 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
     if (lf.A > 1) {
         dim3 grid((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
         rfft_cols_fwd_kernel<<<grid, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(lf), st>>>(a);
+        note_launch(p, "rfft_cols_fwd", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         a.rows_magic = magic_of(2 * lf.tw_rows + 2);
@@ -302,6 +303,7 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
         dim3 grid2(1, (unsigned)batch);
         rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B / 8), rows_fwd_smem(lf), st>>>(a);
     }
+    note_launch(p, "rfft_rows_fwd", st);
     return cudaGetLastError();
 }
 
@@ -317,14 +319,17 @@ cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, f
         a.rows_magic = magic_of(lf.tw_rows);
         dim3 grid((unsigned)(lf.A / lf.tw_rows), (unsigned)batch);
         irfft_rows_kernel<<<grid, threads_for((size_t)lf.B * lf.tw_rows / 8), rows_inv_smem(lf), st>>>(a);
+        note_launch(p, "irfft_rows", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         dim3 grid2((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
         irfft_cols_kernel<<<grid2, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(lf), st>>>(a);
+        note_launch(p, "irfft_cols", st);
     } else {
         a.rows_magic = 0;
         dim3 grid(1, (unsigned)batch);
         irfft_rows_kernel<<<grid, threads_for((size_t)lf.B / 8), rows_inv_smem(lf), st>>>(a);
+        note_launch(p, "irfft_rows", st);
     }
     return cudaGetLastError();
 }
