@@ -110,6 +110,7 @@ int64_t cqt_plan_num_bands(const cqt_plan *plan);
 int64_t cqt_plan_coeff_count(const cqt_plan *plan);   /* sum of M_lambda: complex values per signal */
 int64_t cqt_plan_signal_length(const cqt_plan *plan); /* N */
 int64_t cqt_plan_table_length(const cqt_plan *plan);  /* sum of S_lambda: entries of the g / h tables */
+int cqt_plan_device(const cqt_plan *plan);            /* CUDA device ordinal of the plan, -1 if host-only */
 cqt_status cqt_plan_band_info(const cqt_plan *plan, int64_t band, cqt_band_info *out);
 size_t cqt_plan_workspace_bytes(const cqt_plan *plan, int64_t batch);
 /* Host copies of the fp32 window tables g and h (length cqt_plan_table_length), owned by the plan. */
@@ -139,6 +140,28 @@ cqt_status cqt_plan_read_timing(const cqt_plan *plan, const char **names, float 
  */
 cqt_status cqt_analyse(const cqt_plan *plan, const float *x, int64_t x_stride, int64_t batch,
                        int64_t valid_len, cqt_c64 *c, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Analysis without any allocation by anyone (the paper has no counterpart; this is a deployment aid).
+ * For callers that must not call cudaMalloc: processes running inside a device-memory budget that
+ * was fixed when they started (audio engines with a real-time thread, plug-in hosts, sandboxes),
+ * or code that runs where the allocator is off limits.  Same result as cqt_analyse, but the scratch
+ * comes from a fixed array of CQT_STATIC_WS_BYTES (16 MiB) inside the library image instead of a
+ * caller buffer; every GPU that loads the library holds that array until the process exits.
+ *   - batch is limited by cqt_plan_workspace_bytes(plan, batch) <= cqt_static_workspace_bytes();
+ *     larger requests return CQT_ERR_WORKSPACE and launch nothing.
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current); make that first call before any stream capture begins.
+ *   - All calls share the one array and it keeps whatever the last call left in it; every call
+ *     overwrites what it reads, nothing needs clearing.  Two calls that overlap on the GPU (different
+ *     streams, or different plans) race on it: serialise them.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine, provided event timing
+ *     (cqt_plan_set_timing) is off for the plan.
+ */
+#define CQT_STATIC_WS_BYTES (16u << 20)
+size_t cqt_static_workspace_bytes(void);
+cqt_status cqt_analyse_static_ws(const cqt_plan *plan, const float *x, int64_t x_stride, int64_t batch,
+                                 int64_t valid_len, cqt_c64 *c, void *stream);
 
 /*
  * Synthesis S (Eq. synthesis, packed-synthesis):

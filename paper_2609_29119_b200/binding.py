@@ -43,6 +43,9 @@ EXPORTS = {
     "cqt_plan_coeff_count": (C.c_int64, [C.c_void_p]),
     "cqt_plan_signal_length": (C.c_int64, [C.c_void_p]),
     "cqt_plan_table_length": (C.c_int64, [C.c_void_p]),
+    "cqt_plan_device": (C.c_int, [C.c_void_p]),
+    "cqt_static_workspace_bytes": (C.c_size_t, []),
+    "cqt_analyse_static_ws": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]),
     "cqt_plan_band_info": (C.c_int, [C.c_void_p, C.c_int64, C.POINTER(BandInfo)]),
     "cqt_plan_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int64]),
     "cqt_plan_tables": (C.c_int, [C.c_void_p, C.POINTER(C.POINTER(C.c_float)), C.POINTER(C.POINTER(C.c_float))]),
@@ -188,6 +191,17 @@ class Plan:
         ws = self.workspace(batch) if ws is None else ws
         _check(getattr(self.lib, _fn)(self.handle, x.data_ptr(), stride, batch, vl, out.data_ptr(), ws.data_ptr(),
                                       ws.numel(), _stream_ptr(stream)), _fn)
+        return out
+
+    def analyse_static_ws(self, x, valid_len=None, out=None, stream=None):
+        """cqt_analyse_static_ws: analysis for callers that cannot allocate; scratch is the library's own
+        fixed 16 MiB array (shared by all calls, so overlapping calls race), limited batch."""
+        import torch
+        batch, vl, stride = self._sig(x, valid_len)
+        if out is None:
+            out = torch.empty((batch, self.coeff_count), dtype=torch.complex64, device=x.device)
+        _check(self.lib.cqt_analyse_static_ws(self.handle, x.data_ptr(), stride, batch, vl, out.data_ptr(),
+                                              _stream_ptr(stream)), "cqt_analyse_static_ws")
         return out
 
     def synthesise(self, c, valid_len=None, out=None, ws=None, stream=None, _fn="cqt_synthesise"):

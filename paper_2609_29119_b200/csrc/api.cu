@@ -284,6 +284,7 @@ int64_t cqt_plan_num_bands(const cqt_plan *p) { return p ? (int64_t)p->lay.bands
 int64_t cqt_plan_coeff_count(const cqt_plan *p) { return p ? p->lay.coeff_count : -1; }
 int64_t cqt_plan_signal_length(const cqt_plan *p) { return p ? p->N : -1; }
 int64_t cqt_plan_table_length(const cqt_plan *p) { return p ? p->lay.table_len : -1; }
+int cqt_plan_device(const cqt_plan *p) { return p ? p->device : -1; }
 
 cqt_status cqt_plan_band_info(const cqt_plan *p, int64_t band, cqt_band_info *out) {
     if (!p || !out || band < 0 || band >= (int64_t)p->lay.bands.size()) return CQT_ERR_INVALID_ARG;
