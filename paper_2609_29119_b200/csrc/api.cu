@@ -1,6 +1,7 @@
 // Plan construction and the C ABI of the transform calls (see include/cqt.h).
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
@@ -216,13 +217,39 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     std::vector<int> order(L.bands.size());
     for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L.bands[a].M > L.bands[b].M; });
-    const int64_t smem_cap_elems = (227 * 1024) / 8;
+    int64_t smem_cap_elems = (227 * 1024) / 8;
+    // test hook: a smaller cap sends shorter bands through the two-pass (huge band) kernels
+    if (const char *cap = std::getenv("CQT_TEST_MAX_CTA_ELEMS")) {
+        const long long v = std::atoll(cap);
+        if (v >= 64 && v < smem_cap_elems) smem_cap_elems = v;
+    }
     for (int i : order) {
         const int64_t M = L.bands[i].M;
         const int64_t elems = p->ffts[p->bands[i].fft].generic ? 2 * M : M;
         int c = 0;
         while (M > limits[c]) ++c;
-        if (elems * p->cls[c].items_per_cta > smem_cap_elems) { delete p; return CQT_ERR_UNSUPPORTED; }
+        if (elems * p->cls[c].items_per_cta > smem_cap_elems) {
+            // too long for one CTA: two passes, M = A * B with A the divisor nearest sqrt(M) whose cofactor also plans
+            HugeBand hb;
+            hb.band = i;
+            int64_t bestA = 0;
+            for (int64_t a = 2; a * a <= M; ++a)
+                if (M % a == 0) {
+                    FftPlan t1, t2;
+                    std::vector<float2> scratch_tw;
+                    if (a <= 1600 && M / a <= 1600 && make_fft_plan(a, false, scratch_tw, t1) && !t1.generic &&
+                        make_fft_plan(M / a, false, scratch_tw, t2) && !t2.generic)
+                        bestA = a;
+                }
+            if (!bestA) { delete p; return CQT_ERR_UNSUPPORTED; }
+            hb.A = (int)bestA; hb.B = (int)(M / bestA); hb.TW = 16;
+            hb.fft_A = plan_for(hb.A, false); hb.fft_B = plan_for(hb.B, false);
+            hb.tw_m = append_twiddles(tw, M, hb.log_m_c);
+            hb.scratch_off = p->huge_pitch;
+            p->huge_pitch += (M + 7) / 8 * 8;
+            p->huge.push_back(hb);
+            continue;
+        }
         p->cls[c].work.push_back(i);
         p->cls[c].max_elems = (int)std::max<int64_t>(p->cls[c].max_elems, elems);
         p->cls[c].n_bands++;
@@ -267,6 +294,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     p->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
     if (e == cudaSuccess) chk(configure_band_kernels(*p));
     if (e == cudaSuccess) chk(configure_long_fft_kernels(*p));
+    if (e == cudaSuccess) chk(configure_huge_kernels(*p));
     cudaSetDevice(cur);
     if (e != cudaSuccess) { cqt_plan_destroy(p); return CQT_ERR_CUDA; }
     *out = p;
@@ -301,7 +329,7 @@ cqt_status cqt_plan_band_info(const cqt_plan *p, int64_t band, cqt_band_info *ou
 size_t cqt_plan_workspace_bytes(const cqt_plan *p, int64_t batch) {
     if (!p || batch <= 0) return 0;
     const int64_t t = p->lf.A > 1 ? p->lf.Lp : 0;
-    const int64_t per = std::max<int64_t>(t + p->lf.x_pitch, t + p->y_pitch);
+    const int64_t per = std::max<int64_t>(t + p->lf.x_pitch, t + p->y_pitch) + p->huge_pitch;
     return (size_t)(256 + batch * per * (int64_t)sizeof(float2));
 }
 
@@ -368,7 +396,7 @@ namespace {
 
 struct Call {
     const cqt_plan *p;
-    float2 *T, *second;   // workspace regions
+    float2 *T, *second, *huge;   // workspace regions
     cudaStream_t st;
     int prev_dev;
 };
@@ -383,6 +411,7 @@ cqt_status begin_call(const cqt_plan *p, const void *sig, int64_t stride, int64_
     c.p = p;
     c.T = reinterpret_cast<float2 *>(ws);
     c.second = c.T + (p->lf.A > 1 ? batch * p->lf.Lp : 0);
+    c.huge = c.second + batch * std::max<int64_t>(p->lf.x_pitch, p->y_pitch);
     c.st = reinterpret_cast<cudaStream_t>(stream);
     if (cudaGetDevice(&c.prev_dev) != cudaSuccess) return CQT_ERR_CUDA;
     if (c.prev_dev != p->device && cudaSetDevice(p->device) != cudaSuccess) return CQT_ERR_CUDA;
@@ -401,6 +430,7 @@ cqt_status run_analysis_form(const cqt_plan *p, const float *table, const float 
     cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
     if (s != CQT_OK) return s;
     cudaError_t e = launch_rfft_forward(*p, x, x_stride, batch, valid_len, k.T, k.second, k.st);
+    if (e == cudaSuccess) e = launch_huge_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), k.huge, batch, k.st);
     if (e == cudaSuccess) e = launch_bands_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), batch, k.st);
     return end_call(k, e);
 }
@@ -410,7 +440,8 @@ cqt_status run_synthesis_form(const cqt_plan *p, const float *table, bool fold, 
     Call k;
     cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
     if (s != CQT_OK) return s;
-    cudaError_t e = launch_bands_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, batch, k.st);
+    cudaError_t e = launch_huge_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, k.huge, batch, k.st);
+    if (e == cudaSuccess) e = launch_bands_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, batch, k.st);
     if (e == cudaSuccess) e = launch_rfft_inverse(*p, k.second, k.T, x, x_stride, batch, valid_len, k.st);
     return end_call(k, e);
 }

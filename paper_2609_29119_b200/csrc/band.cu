@@ -97,23 +97,22 @@ __global__ void __launch_bounds__(WARP ? 256 : 512) bands_to_spectrum_kernel(Ban
     float2 *alt = buf + br.M;
     const int M = br.M;
     const float2 *in = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
-    for (int n = tid; n < M; n += nthr) buf[n] = __ldg(in + n);
+    // adjoint of analysis, sidebands: U[m] + conj U[-m] is the DFT of 2 Re c
+    const bool fold = a.fold && br.side != 0;
+    for (int n = tid; n < M; n += nthr) {
+        float2 v = __ldg(in + n);
+        if (fold) v = make_float2(2.f * v.x, 0.f);
+        buf[n] = v;
+    }
     Sync::sync();
     fft_dif<-1, Sync, false>(buf, alt, 1, 1, 0u, fp, a.tw, tid, nthr);
     const float *tab = a.table + br.tab_off;
     float2 *Y = a.Y + (long long)ch * a.y_pitch + br.y_off;
-    const bool fold = a.fold && br.side != 0;
     for (int i = tid; i < br.n_in; i += nthr) {
         const int j = br.j_lo + i;
         const int d = br.d0 + j;
         const int m = d < 0 ? d + M : d;
-        float2 u = buf[dif_pos(fp, m)];
-        if (fold) {
-            const int m2 = d > 0 ? M - d : -d;
-            const float2 u2 = buf[dif_pos(fp, m2)];
-            u.x += u2.x;
-            u.y -= u2.y;
-        }
+        const float2 u = buf[dif_pos(fp, m)];
         const float h = __ldg(tab + j);
         Y[i] = make_float2(h * u.x, h * u.y);
     }

@@ -33,6 +33,15 @@ struct LongFft {
     int64_t x_pitch = 0;          // elements per signal of the half-spectrum buffer (Lp + 1 rounded up)
 };
 
+// A band too long for one CTA: M = A * B, two passes through a scratch row of M complex values.
+struct HugeBand {
+    int band = 0;
+    int A = 0, B = 0, TW = 16;
+    int fft_A = -1, fft_B = -1;
+    int tw_m = 0, log_m_c = 0;
+    int64_t scratch_off = 0;   // into one signal's huge-band scratch row
+};
+
 struct DevicePlan {
     BandRec *bands = nullptr;
     FftPlan *ffts = nullptr;
@@ -57,6 +66,8 @@ struct cqt_plan {
     int64_t y_pitch = 0;
     cqt::LongFft lf;
     cqt::BandClass cls[cqt::kNumClasses];
+    std::vector<cqt::HugeBand> huge;
+    int64_t huge_pitch = 0;            // scratch elements per signal for the huge bands
     cqt::DevicePlan d;
     int max_smem_optin = 0;
     int sm_count = 0;
@@ -89,5 +100,12 @@ cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, co
 cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool fold_sidebands, const float2 *c,
                                      float2 *Y, int64_t batch, cudaStream_t st);
 cudaError_t configure_band_kernels(const cqt_plan &p);
+
+// band_huge.cu
+cudaError_t launch_huge_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c, float2 *scratch,
+                                      int64_t batch, cudaStream_t st);
+cudaError_t launch_huge_to_spectrum(const cqt_plan &p, const float *table, bool fold, const float2 *c, float2 *Y,
+                                    float2 *scratch, int64_t batch, cudaStream_t st);
+cudaError_t configure_huge_kernels(const cqt_plan &p);
 
 }  // namespace cqt
