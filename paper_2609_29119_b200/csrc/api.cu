@@ -84,11 +84,16 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp) {
         fp.stride[j] = (int32_t)(n_cur / radices[j]);
         fp.rmagic[j] = magic_of((uint32_t)radices[j]);
         fp.smagic[j] = magic_of((uint32_t)fp.stride[j]);
+        const int64_t kd = j == 0 ? 1 : fp.stride[0] / n_cur;
+        fp.k1div[j] = (int32_t)kd;
+        fp.k1magic[j] = magic_of((uint32_t)kd);
         n_cur /= radices[j];
     }
     int logC;
     fp.tw_off = append_twiddles(tw, M, logC);
     fp.logC = logC;
+    fp.tw_count = (int32_t)((1ll << logC) + (M + (1ll << logC) - 1) / (1ll << logC));
+    fp.pad_delta = (fp.nstages > 1 && (fp.stride[0] % 2 == 0)) ? 1 : 0;
     return true;
 }
 
@@ -208,8 +213,10 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         if (br.fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
     }
     // ---- launch classes by band length
-    const int limits[kNumClasses] = {128, 2048, 8192, 1 << 30};
-    const int threads[kNumClasses] = {256, 128, 256, 512};
+    // class 0: one warp per item, 8 items per CTA; the others one CTA per item, sized so that several CTAs
+    // share an SM (64 registers per thread) except for the longest bands, which fill its shared memory
+    const int limits[kNumClasses] = {128, 1024, 4096, 13500, 1 << 30};
+    const int threads[kNumClasses] = {256, 64, 256, 512, 1024};
     for (int c = 0; c < kNumClasses; ++c) {
         p->cls[c].threads = threads[c];
         p->cls[c].items_per_cta = c == 0 ? 8 : 1;
@@ -225,7 +232,9 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     }
     for (int i : order) {
         const int64_t M = L.bands[i].M;
-        const int64_t elems = p->ffts[p->bands[i].fft].generic ? 2 * M : M;
+        // shared memory per item: padded buffer + two-level twiddle table (two buffers for generic radices)
+        const FftPlan &bf = p->ffts[p->bands[i].fft];
+        const int64_t elems = bf.generic ? 2 * M : M + 16 + bf.tw_count;
         int c = 0;
         while (M > limits[c]) ++c;
         if (elems * p->cls[c].items_per_cta > smem_cap_elems) {

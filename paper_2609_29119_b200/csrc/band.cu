@@ -32,6 +32,7 @@ struct BandArgs {
     long long y_pitch;
 };
 
+// THREADS / MINB: launch bounds of the class (64 registers per thread when THREADS * MINB = 1024 ... 2048)
 template <bool WARP>
 struct Group {
     __device__ static int tid() { return WARP ? (threadIdx.x & 31) : threadIdx.x; }
@@ -42,8 +43,8 @@ struct Group {
 
 extern __shared__ float2 smem_band[];
 
-template <bool WARP>
-__global__ void __launch_bounds__(WARP ? 256 : 512) bands_from_spectrum_kernel(BandArgs a) {
+template <int THREADS, int MINB, bool WARP>
+__global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
     using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
     const int item = G::item();
@@ -53,38 +54,43 @@ __global__ void __launch_bounds__(WARP ? 256 : 512) bands_from_spectrum_kernel(B
     const int ch = item % a.batch;
     const FftPlan &fp = a.ffts[br.fft];
     float2 *buf = smem_band + (size_t)G::slot() * a.max_elems;
-    float2 *alt = buf + br.M;
     const float2 *X = a.spec + (long long)ch * a.spec_pitch;
     const float *tab = a.table + br.tab_off;
     const int M = br.M, half = a.N >> 1;
     const int last_pos = br.d0 + br.S - 1;   // largest offset (>= 0)
     const int first_neg = M + br.d0;          // slot of the most negative offset
-    for (int m = tid; m < M; m += nthr) {
+    // slot m holds tab[d] X[kc + d] with d = m (m <= last_pos) or m - M (m >= first_neg), else zero
+    auto load = [&](int m, int) -> float2 {
         int d;
-        bool in = true;
         if (m <= last_pos) d = m;
         else if (m >= first_neg) d = m - M;
-        else { in = false; d = 0; }
-        float2 v = make_float2(0.f, 0.f);
-        if (in) {
-            const float g = __ldg(tab + (d - br.d0));
-            int k = br.kc + d;
-            float2 xv;
-            if (k < 0) xv = cconj(__ldg(X + (-k)));
-            else if (k > half) xv = cconj(__ldg(X + (a.N - k)));
-            else xv = __ldg(X + k);
-            v = make_float2(g * xv.x, g * xv.y);
-        }
-        buf[m] = v;
-    }
-    Sync::sync();
-    fft_dif<+1, Sync, false>(buf, alt, 1, 1, 0u, fp, a.tw, tid, nthr);
+        else return make_float2(0.f, 0.f);
+        const float g = __ldg(tab + (d - br.d0));
+        const int k = br.kc + d;
+        float2 xv;
+        if (k < 0) xv = cconj(__ldg(X + (-k)));
+        else if (k > half) xv = cconj(__ldg(X + (a.N - k)));
+        else xv = __ldg(X + k);
+        return make_float2(g * xv.x, g * xv.y);
+    };
     float2 *out = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
-    for (int n = tid; n < M; n += nthr) out[n] = buf[dif_pos(fp, n)];
+    if (fp.generic) {
+        float2 *alt = buf + M;
+        for (int m = tid; m < M; m += nthr) buf[m] = load(m, 0);
+        Sync::sync();
+        fft_dif<+1, Sync, false>(buf, alt, 1, 1, 0u, fp, a.tw, tid, nthr);
+        for (int n = tid; n < M; n += nthr) out[n] = buf[dif_pos(fp, n)];
+        return;
+    }
+    float2 *tws = buf + M + 16;
+    if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
+    const Tile t{buf, 1, 1, 0u};
+    auto store = [&](int n, int, float2 v) { out[n] = v; };
+    fft_fused<+1, Sync, false, true, false, true, false>(t, fp, tws, load, store, tid, nthr);
 }
 
-template <bool WARP>
-__global__ void __launch_bounds__(WARP ? 256 : 512) bands_to_spectrum_kernel(BandArgs a) {
+template <int THREADS, int MINB, bool WARP>
+__global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
     using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
     const int item = G::item();
@@ -94,28 +100,41 @@ __global__ void __launch_bounds__(WARP ? 256 : 512) bands_to_spectrum_kernel(Ban
     const int ch = item % a.batch;
     const FftPlan &fp = a.ffts[br.fft];
     float2 *buf = smem_band + (size_t)G::slot() * a.max_elems;
-    float2 *alt = buf + br.M;
     const int M = br.M;
     const float2 *in = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
     // adjoint of analysis, sidebands: U[m] + conj U[-m] is the DFT of 2 Re c
     const bool fold = a.fold && br.side != 0;
-    for (int n = tid; n < M; n += nthr) {
+    auto load = [&](int n, int) -> float2 {
         float2 v = __ldg(in + n);
         if (fold) v = make_float2(2.f * v.x, 0.f);
-        buf[n] = v;
-    }
-    Sync::sync();
-    fft_dif<-1, Sync, false>(buf, alt, 1, 1, 0u, fp, a.tw, tid, nthr);
+        return v;
+    };
     const float *tab = a.table + br.tab_off;
     float2 *Y = a.Y + (long long)ch * a.y_pitch + br.y_off;
-    for (int i = tid; i < br.n_in; i += nthr) {
-        const int j = br.j_lo + i;
-        const int d = br.d0 + j;
-        const int m = d < 0 ? d + M : d;
-        const float2 u = buf[dif_pos(fp, m)];
+    const int last_pos = br.d0 + br.S - 1, first_neg = M + br.d0;
+    // slot m -> offset d -> support index j -> entry j - j_lo of the band's weighted-bin run
+    auto store = [&](int m, int, float2 u) {
+        int d;
+        if (m <= last_pos) d = m;
+        else if (m >= first_neg) d = m - M;
+        else return;
+        const int j = d - br.d0, i = j - br.j_lo;
+        if (i < 0 || i >= br.n_in) return;
         const float h = __ldg(tab + j);
         Y[i] = make_float2(h * u.x, h * u.y);
+    };
+    if (fp.generic) {
+        float2 *alt = buf + M;
+        for (int n = tid; n < M; n += nthr) buf[n] = load(n, 0);
+        Sync::sync();
+        fft_dif<-1, Sync, false>(buf, alt, 1, 1, 0u, fp, a.tw, tid, nthr);
+        for (int m = tid; m < M; m += nthr) store(m, 0, buf[dif_pos(fp, m)]);
+        return;
     }
+    float2 *tws = buf + M + 16;
+    if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
+    const Tile t{buf, 1, 1, 0u};
+    fft_fused<-1, Sync, false, true, false, true, false>(t, fp, tws, load, store, tid, nthr);
 }
 
 static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *table, int64_t batch) {
@@ -134,31 +153,42 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
     return a;
 }
 
-template <class K>
-static cudaError_t launch_class(const cqt_plan &p, const char *name, K warp_kernel, K block_kernel, const BandClass &c,
-                                BandArgs &a, cudaStream_t st) {
+// one instantiation per length class: threads per CTA and CTAs per SM the registers must allow
+#define CQT_CLASS_TABLE(X) X(0, 256, 2, true) X(1, 64, 16, false) X(2, 256, 4, false) X(3, 512, 2, false) X(4, 1024, 1, false)
+
+template <bool ANALYSIS>
+static const void *class_kernel(int cls) {
+#define X(C, T, B, W) \
+    if (cls == C) return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W> : (const void *)bands_to_spectrum_kernel<T, B, W>;
+    CQT_CLASS_TABLE(X)
+#undef X
+    return nullptr;
+}
+
+template <bool ANALYSIS>
+static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, BandArgs &a, cudaStream_t st) {
+    const BandClass &c = p.cls[cls];
     if (c.n_bands == 0) return cudaSuccess;
     const long long items = (long long)c.n_bands * a.batch;
     const size_t smem = (size_t)c.max_elems * c.items_per_cta * sizeof(float2);
     const long long grid = (items + c.items_per_cta - 1) / c.items_per_cta;
-    if (c.items_per_cta > 1)
-        warp_kernel<<<(unsigned)grid, c.threads, smem, st>>>(a);
-    else
-        block_kernel<<<(unsigned)grid, c.threads, smem, st>>>(a);
+    void *args[] = {&a};
+    cudaError_t e = cudaLaunchKernel(class_kernel<ANALYSIS>(cls), dim3((unsigned)grid), dim3(c.threads), args, smem, st);
     note_launch(p, name, st);
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
                                        int64_t batch, cudaStream_t st) {
+    static const char *names[kNumClasses] = {"bands_from_spectrum/class0", "bands_from_spectrum/class1",
+                                              "bands_from_spectrum/class2", "bands_from_spectrum/class3",
+                                              "bands_from_spectrum/class4"};
     for (int i = kNumClasses - 1; i >= 0; --i) {   // longest bands first
         BandArgs a = make_args(p, p.cls[i], table, batch);
         a.spec = X;
         a.spec_pitch = p.lf.x_pitch;
         a.coef = c;
-        static const char *names[kNumClasses] = {"bands_from_spectrum/class0", "bands_from_spectrum/class1",
-                                                  "bands_from_spectrum/class2", "bands_from_spectrum/class3"};
-        cudaError_t e = launch_class(p, names[i], bands_from_spectrum_kernel<true>, bands_from_spectrum_kernel<false>, p.cls[i], a, st);
+        cudaError_t e = launch_class<true>(p, i, names[i], a, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -166,31 +196,30 @@ cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, co
 
 cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool fold_sidebands, const float2 *c,
                                      float2 *Y, int64_t batch, cudaStream_t st) {
+    static const char *names[kNumClasses] = {"bands_to_spectrum/class0", "bands_to_spectrum/class1",
+                                              "bands_to_spectrum/class2", "bands_to_spectrum/class3",
+                                              "bands_to_spectrum/class4"};
     for (int i = kNumClasses - 1; i >= 0; --i) {
         BandArgs a = make_args(p, p.cls[i], table, batch);
         a.coef = const_cast<float2 *>(c);
         a.Y = Y;
         a.fold = fold_sidebands ? 1 : 0;
-        static const char *names[kNumClasses] = {"bands_to_spectrum/class0", "bands_to_spectrum/class1",
-                                                  "bands_to_spectrum/class2", "bands_to_spectrum/class3"};
-        cudaError_t e = launch_class(p, names[i], bands_to_spectrum_kernel<true>, bands_to_spectrum_kernel<false>, p.cls[i], a, st);
+        cudaError_t e = launch_class<false>(p, i, names[i], a, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
 }
 
 cudaError_t configure_band_kernels(const cqt_plan &p) {
-    size_t need = 0;
     for (int i = 0; i < kNumClasses; ++i) {
         const size_t s = (size_t)p.cls[i].max_elems * p.cls[i].items_per_cta * sizeof(float2);
-        if (s > need) need = s;
+        if (s <= 48 * 1024) continue;
+        cudaError_t e = cudaFuncSetAttribute(class_kernel<true>(i), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(class_kernel<false>(i), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
+        if (e != cudaSuccess) return e;
     }
-    if (need <= 48 * 1024) return cudaSuccess;
-    cudaError_t e;
-    e = cudaFuncSetAttribute(bands_from_spectrum_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(bands_to_spectrum_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
-    return e;
+    return cudaSuccess;
 }
 
 }  // namespace cqt

@@ -158,4 +158,258 @@ __device__ void fft_dif(float2 *buf, float2 *alt, int pitch, int ncols, uint32_t
     }
 }
 
+// ======================================================================================
+// Fused engine.  The first stage reads its operands through a caller functor (straight from
+// global memory), the last stage hands its results to a caller functor (straight to global
+// memory), the stages in between run in shared memory.  Twiddles: one two-level lookup per
+// butterfly from a shared-memory copy of the plan's table, the powers w^2 .. w^(R-1) are formed
+// in registers by balanced products (depth <= log2 R, so rounding grows with the depth only).
+// ======================================================================================
+
+// copies the two-level table of a plan into shared memory (caller synchronises afterwards)
+__device__ __forceinline__ void stage_twiddles(float2 *dst, const float2 *__restrict__ tw_base, const FftPlan &fp, int tid,
+                                               int nthr) {
+    const float2 *src = tw_base + fp.tw_off;
+    for (int i = tid; i < fp.tw_count; i += nthr) dst[i] = __ldg(src + i);
+}
+
+__device__ __forceinline__ float2 twiddle_s(const float2 *tw, int logC, uint32_t y) {
+    const uint32_t C = 1u << logC;
+    return cmul(tw[y & (C - 1)], tw[C + (y >> logC)]);
+}
+
+template <int R>
+__device__ __forceinline__ void apply_twiddle_powers(float2 w1, float (&re)[R], float (&im)[R]) {
+    float wr[R], wi[R];
+    wr[0] = 1.f; wi[0] = 0.f;
+    wr[1] = w1.x; wi[1] = w1.y;
+#pragma unroll
+    for (int q = 2; q < R; ++q) {
+        const int a = (q + 1) / 2, b = q / 2;
+        wr[q] = fmaf(wr[a], wr[b], -wi[a] * wi[b]);
+        wi[q] = fmaf(wr[a], wi[b], wi[a] * wr[b]);
+    }
+#pragma unroll
+    for (int q = 1; q < R; ++q) {
+        const float x = re[q], y = im[q];
+        re[q] = fmaf(x, wr[q], -y * wi[q]);
+        im[q] = fmaf(x, wi[q], y * wr[q]);
+    }
+}
+
+struct Tile {
+    float2 *buf;
+    int pitch;             // elements between consecutive positions
+    int ncols;             // interleaved columns
+    uint32_t ncols_magic;
+};
+
+// first stage: operands from load(pos, col); results to shared memory.
+// COLFAST: consecutive threads take consecutive columns, else consecutive butterflies.
+template <int R, int SIGN, bool PAD, bool COLFAST, class Sync, class Load>
+__device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
+    const int s = fp.stride[0];
+    const int total = s * t.ncols;
+    const int spad = PAD ? s + fp.pad_delta : s;
+    // every thread of the group runs every round: the first round contains the barrier that makes the
+    // staged twiddle table visible, placed after the operand loads so both are in flight together
+    for (int base = 0; base < total; base += nthr) {
+        const int w = base + tid;
+        const bool active = w < total;
+        uint32_t b = 0, col = 0;
+        if (active) {
+            if (t.ncols == 1) { b = w; }
+            else if (COLFAST) { b = fastdiv(w, t.ncols_magic, t.ncols); col = w - b * t.ncols; }
+            else { col = fastdiv(w, fp.smagic[0], s); b = w - col * s; }
+        }
+        float re[R], im[R];
+        if (active) {
+#pragma unroll
+            for (int q = 0; q < R; ++q) {
+                const float2 v = load((int)(b + q * s), (int)col);
+                re[q] = v.x; im[q] = v.y;
+            }
+            if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
+        }
+        if (base == 0) Sync::sync();
+        if (active) {
+            float2 w1 = twiddle_s(tw, fp.logC, b);
+            if (SIGN > 0) w1.y = -w1.y;
+            apply_twiddle_powers<R>(w1, re, im);
+            float2 *p = t.buf + (size_t)b * t.pitch + col;
+#pragma unroll
+            for (int q = 0; q < R; ++q) p[(size_t)q * spad * t.pitch] = make_float2(re[q], im[q]);
+        }
+    }
+}
+
+template <int R, int SIGN, bool PAD>
+__device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, const float2 *tw, int j, int n_cur, int tmul,
+                                             int tid, int nthr) {
+    const int s = fp.stride[j];
+    const int total = (fp.M / R) * t.ncols;
+    for (int w = tid; w < total; w += nthr) {
+        const uint32_t b = fastdiv(w, t.ncols_magic, t.ncols);
+        const uint32_t col = w - b * t.ncols;
+        const uint32_t blk = fastdiv(b, fp.smagic[j], s);
+        const uint32_t np = b - blk * s;
+        uint32_t pos = blk * n_cur + np;
+        if (PAD) pos += fp.pad_delta ? fastdiv(blk, fp.k1magic[j], fp.k1div[j]) : 0u;
+        float2 *p = t.buf + (size_t)pos * t.pitch + col;
+        const int step = s * t.pitch;
+        float re[R], im[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) {
+            const float2 v = p[q * step];
+            re[q] = v.x; im[q] = v.y;
+        }
+        if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
+        float2 w1 = twiddle_s(tw, fp.logC, np * tmul);
+        if (SIGN > 0) w1.y = -w1.y;
+        apply_twiddle_powers<R>(w1, re, im);
+#pragma unroll
+        for (int q = 0; q < R; ++q) p[q * step] = make_float2(re[q], im[q]);
+    }
+}
+
+// last stage (stride 1): operands from shared memory, result k of column col to store(k, col, value).
+// REV: thread index = low digits of k (consecutive threads store consecutive k), else thread index =
+// butterfly position.  COLFAST as above.
+template <int R, int SIGN, bool PAD, bool REV, bool COLFAST, class Store>
+__device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Store store, int tid, int nthr) {
+    const int nb = fp.M / R;
+    const int total = nb * t.ncols;
+    const int d = fp.nstages;
+    for (int w = tid; w < total; w += nthr) {
+        uint32_t u, col;
+        if (t.ncols == 1) { u = w; col = 0; }
+        else if (COLFAST) { u = fastdiv(w, t.ncols_magic, t.ncols); col = w - u * t.ncols; }
+        else { col = (uint32_t)w / (uint32_t)nb; u = w - col * nb; }
+        uint32_t b, klow;
+        if (REV) {           // u = k_0 + r_0 (k_1 + ...)  ->  b = ((k_0 r_1 + k_1) r_2 + ...)
+            klow = u;
+            uint32_t rem = u;
+            // Horner over the digits, most significant first
+            b = 0;
+#pragma unroll 1
+            for (int j = 0; j < d - 1; ++j) {
+                const uint32_t r = fp.radix[j];
+                const uint32_t qd = __umulhi(rem, fp.rmagic[j]);
+                b = b * r + (rem - qd * r);
+                rem = qd;
+            }
+        } else {             // u = b  ->  k_low = k_0 + r_0 (k_1 + r_1 (...)), digits of b least significant first
+            b = u; klow = 0;
+            uint32_t rem = u;
+#pragma unroll 1
+            for (int j = d - 2; j >= 0; --j) {
+                const uint32_t r = fp.radix[j];
+                const uint32_t qd = __umulhi(rem, fp.rmagic[j]);
+                klow = klow * r + (rem - qd * r);
+                rem = qd;
+            }
+        }
+        uint32_t pos = b * R;
+        if (PAD) pos += fp.pad_delta ? fastdiv(b, fp.k1magic[d - 1], fp.k1div[d - 1]) : 0u;
+        const float2 *p = t.buf + (size_t)pos * t.pitch + col;
+        float re[R], im[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) {
+            const float2 v = p[q * t.pitch];
+            re[q] = v.x; im[q] = v.y;
+        }
+        if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
+#pragma unroll
+        for (int q = 0; q < R; ++q) store((int)(klow + q * nb), (int)col, make_float2(re[q], im[q]));
+    }
+}
+
+// single-stage transform (M = R): no shared memory at all
+template <int R, int SIGN, class Load, class Store>
+__device__ __forceinline__ void only_stage(const Tile &t, Load load, Store store, int tid, int nthr) {
+    for (int col = tid; col < t.ncols; col += nthr) {
+        float re[R], im[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) {
+            const float2 v = load(q, col);
+            re[q] = v.x; im[q] = v.y;
+        }
+        if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
+#pragma unroll
+        for (int q = 0; q < R; ++q) store(q, col, make_float2(re[q], im[q]));
+    }
+}
+
+#define CQT_RADIX_CASES_ALL(X) X(2) X(3) X(4) X(5) X(6) X(8) X(9) X(10) X(12) X(15) X(16)
+#define CQT_RADIX_CASES_POW2(X) X(2) X(4) X(8) X(16) X(32)
+
+// Runs the first `nrun` stages of the plan (nrun = nstages: the whole transform with the last stage fused
+// into `store`; nrun = nstages - 1... not offered: use fft_fused_keep for "results stay in shared memory").
+// Requires a non-generic plan.  tw = shared-memory copy of the plan's two-level table, written by the
+// caller (stage_twiddles) WITHOUT a barrier after it: the first stage synchronises once its operand loads
+// are issued.  The routine synchronises between stages, not at the end.
+template <int SIGN, class Sync, bool POW2, bool PAD, bool COLFAST_IN, bool REV, bool COLFAST_OUT, class Load, class Store>
+__device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, Store store, int tid, int nthr) {
+    const int d = fp.nstages;
+    if (d == 1) {
+#define X(RR) case RR: only_stage<RR, SIGN>(t, load, store, tid, nthr); break;
+        if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+#undef X
+        return;
+    }
+#define X(RR) case RR: first_stage<RR, SIGN, PAD, COLFAST_IN, Sync>(t, fp, tw, load, tid, nthr); break;
+    if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
+    else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+#undef X
+    Sync::sync();
+    int n_cur = fp.stride[0], tmul = fp.radix[0];
+#pragma unroll 1
+    for (int j = 1; j < d - 1; ++j) {
+#define X(RR) case RR: middle_stage<RR, SIGN, PAD>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+        if (POW2) { switch (fp.radix[j]) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.radix[j]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+#undef X
+        Sync::sync();
+        n_cur = fp.stride[j];
+        tmul *= fp.radix[j];
+    }
+#define X(RR) case RR: last_stage<RR, SIGN, PAD, REV, COLFAST_OUT>(t, fp, store, tid, nthr); break;
+    if (POW2) { switch (fp.radix[d - 1]) { CQT_RADIX_CASES_POW2(X) default: break; } }
+    else { switch (fp.radix[d - 1]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+#undef X
+}
+
+// Same, but every stage after the first runs in shared memory and the results stay there
+// (digit-reversed positions, see dif_pos); ends with a sync.
+template <int SIGN, class Sync, bool POW2, bool COLFAST_IN, class Load>
+__device__ void fft_fused_keep(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
+    const int d = fp.nstages;
+    if (d == 1) {
+        auto keep = [&](int k, int col, float2 v) { t.buf[(size_t)k * t.pitch + col] = v; };
+#define X(RR) case RR: only_stage<RR, SIGN>(t, load, keep, tid, nthr); break;
+        if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+#undef X
+        Sync::sync();
+        return;
+    }
+#define X(RR) case RR: first_stage<RR, SIGN, false, COLFAST_IN, Sync>(t, fp, tw, load, tid, nthr); break;
+    if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
+    else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+#undef X
+    Sync::sync();
+    int n_cur = fp.stride[0], tmul = fp.radix[0];
+#pragma unroll 1
+    for (int j = 1; j < d; ++j) {
+#define X(RR) case RR: middle_stage<RR, SIGN, false>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+        if (POW2) { switch (fp.radix[j]) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.radix[j]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+#undef X
+        Sync::sync();
+        n_cur = fp.stride[j];
+        tmul *= fp.radix[j];
+    }
+}
+
 }  // namespace cqt

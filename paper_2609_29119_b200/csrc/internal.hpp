@@ -11,7 +11,7 @@
 
 namespace cqt {
 
-constexpr int kNumClasses = 4;
+constexpr int kNumClasses = 5;
 
 // Launch shape of one band-length class.
 struct BandClass {
