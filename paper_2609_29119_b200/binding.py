@@ -162,6 +162,10 @@ class Plan:
             self._ws = torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}")
         return self._ws
 
+    def check(self) -> int:
+        """cqt_plan_check: 0, or -7 if a debug-bounds build recorded an out-of-range index (printed to stderr)."""
+        return int(self.lib.cqt_plan_check(self.handle))
+
     def launch_count(self) -> int:
         return int(self.lib.cqt_plan_launch_count(self.handle))
 

@@ -31,8 +31,19 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    """debug_bounds=True (or CQT_DEBUG_BOUNDS=1 in the environment) compiles the index self-checks in: an
+    out-of-range index is recorded for cqt_plan_check and the access skipped (slower; for debugging only)."""
+    debug_bounds = debug_bounds or os.environ.get("CQT_DEBUG_BOUNDS") == "1"
+    flags_extra = ["-DCQT_DEBUG_BOUNDS"] if debug_bounds else []
+    stamp = os.path.join(OBJ, "debug_bounds.stamp")
     os.makedirs(OBJ, exist_ok=True)
+    if debug_bounds != os.path.exists(stamp):
+        force = True
+        if debug_bounds:
+            open(stamp, "w").close()
+        else:
+            os.unlink(stamp)
     hdrs = [os.path.join(CSRC, h) for h in HEADERS]
     nvcc = _nvcc()
     jobs = []
@@ -42,7 +53,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(OBJ, os.path.splitext(s)[0] + ".o")
         objs.append(obj)
         if force or _stale(obj, [src] + hdrs):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-x", "cu", "-c", src, "-o", obj]
+            cmd = [nvcc] + NVCC_FLAGS + flags_extra + (["-Xptxas", "-v"] if verbose else []) + ["-x", "cu", "-c", src, "-o", obj]
             jobs.append(cmd)
     if jobs:
         with cf.ThreadPoolExecutor(max_workers=min(8, len(jobs))) as ex:
@@ -61,4 +72,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

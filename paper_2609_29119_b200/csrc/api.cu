@@ -1,6 +1,7 @@
 // Plan construction and the C ABI of the transform calls (see include/cqt.h).
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <map>
@@ -36,7 +37,7 @@ int append_twiddles(std::vector<float2> &tw, int64_t n, int &logC) {
 }
 
 const int kBandRadices[] = {16, 15, 12, 10, 9, 8, 6, 5, 4, 3, 2};
-const int kPow2Radices[] = {32, 16, 8, 4, 2};
+const int kPow2Radices[] = {16, 8, 4, 2};
 
 // fewest stages, then smallest largest radix
 bool best_split(int64_t m, const int *radices, int nr, std::map<int64_t, std::vector<int>> &memo, std::vector<int> &out) {
@@ -73,7 +74,7 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp) {
     }
     std::map<int64_t, std::vector<int>> memo;
     std::vector<int> radices;
-    if (!best_split(smooth, pow2 ? kPow2Radices : kBandRadices, pow2 ? 5 : 11, memo, radices)) return false;
+    if (!best_split(smooth, pow2 ? kPow2Radices : kBandRadices, pow2 ? 4 : 11, memo, radices)) return false;
     if (rest > 1) { radices.insert(radices.begin(), (int)rest); fp.generic = 1; }
     if (radices.empty()) radices.push_back(1);
     if ((int)radices.size() > kMaxStages) return false;
@@ -114,7 +115,7 @@ void free_device(cqt_plan *p) {
     cudaFree(p->d.bands); cudaFree(p->d.ffts); cudaFree(p->d.tw);
     cudaFree(p->d.tab_analysis); cudaFree(p->d.tab_synthesis);
     cudaFree(p->d.tab_analysis_adj); cudaFree(p->d.tab_synthesis_adj);
-    cudaFree(p->d.cover); cudaFree(p->d.span);
+    cudaFree(p->d.cover); cudaFree(p->d.dbg);
     for (auto &c : p->cls) cudaFree(c.d_work);
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     cudaSetDevice(cur);
@@ -169,7 +170,10 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     p->g32.resize(L.table_len);
     p->h32.resize(L.table_len);
     for (int64_t i = 0; i < L.table_len; ++i) { p->g32[i] = (float)L.g[i]; p->h32[i] = (float)L.h[i]; }
-    p->y_pitch = (L.y_len + 7) / 8 * 8;
+    p->y_planes = 1;
+    for (int64_t k = 0; k <= N / 2; ++k) p->y_planes = std::max(p->y_planes, (int)L.cover_n[k]);
+    p->y_plane = (N / 2 + 1 + 7) / 8 * 8;
+    p->y_pitch = p->y_plane * p->y_planes;
 
     // ---- transform-length plans and twiddles
     std::vector<float2> tw;
@@ -195,9 +199,13 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     lf.fft_B = plan_for(lf.B, true);
     lf.fft_A = lf.A > 1 ? plan_for(lf.A, true) : lf.fft_B;
     lf.tw_lp = append_twiddles(tw, lf.Lp, lf.log_lp_c);
+    lf.n_lp = (int)tw.size() - lf.tw_lp;
     lf.tw_n = append_twiddles(tw, N, lf.log_n_c);
-    lf.tw_rows = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.B <= 512 ? 16 : 8, lf.A / 2);
-    lf.tw_cols = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.A <= 1024 ? 16 : 8, lf.B);
+    lf.n_n = (int)tw.size() - lf.tw_n;
+    // tile widths chosen so that two CTAs of the row kernels (three of the column kernels) share an SM
+    lf.tw_rows = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.B <= 512 ? 8 : 4, lf.A / 2);
+    lf.tw_rows_inv = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.B <= 512 ? 16 : 8, lf.A);
+    lf.tw_cols = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.A <= 512 ? 16 : 8, lf.B);
     lf.x_pitch = (lf.Lp + 1 + 7) / 8 * 8;
 
     // ---- band records
@@ -206,7 +214,8 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         const HostBand &hb = L.bands[i];
         BandRec &br = p->bands[i];
         br.kc = (int32_t)hb.kc; br.d0 = (int32_t)hb.d0; br.S = (int32_t)hb.S; br.M = (int32_t)hb.M;
-        br.tab_off = (int32_t)hb.tab_off; br.coeff_off = (int32_t)hb.coeff_off; br.y_off = (int32_t)hb.y_off;
+        br.tab_off = (int32_t)hb.tab_off; br.coeff_off = (int32_t)hb.coeff_off;
+        br.y_off = (int32_t)((int64_t)(i % p->y_planes) * p->y_plane);
         br.j_lo = (int32_t)hb.j_lo; br.n_in = (int32_t)hb.n_in; br.side = hb.side;
         br.inv_M = (float)(1.0 / (double)hb.M);
         br.fft = plan_for(hb.M, false);
@@ -263,16 +272,29 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         p->cls[c].max_elems = (int)std::max<int64_t>(p->cls[c].max_elems, elems);
         p->cls[c].n_bands++;
     }
+    if (std::getenv("CQT_VERBOSE_PLAN")) {
+        std::fprintf(stderr, "cqt plan: N %lld Lp %lld A %lld B %lld fftA %d fftB %d tw_rows %d tw_rows_inv %d tw_cols %d n_lp %d n_n %d "
+                     "logC %d %d planes %d y_plane %lld bands %zu ffts %zu tw %zu\n", (long long)N, (long long)lf.Lp,
+                     (long long)lf.A, (long long)lf.B, lf.fft_A, lf.fft_B, lf.tw_rows, lf.tw_rows_inv, lf.tw_cols, lf.n_lp,
+                     lf.n_n, lf.log_lp_c, lf.log_n_c, p->y_planes, (long long)p->y_plane, p->bands.size(), p->ffts.size(), tw.size());
+        for (int f : {lf.fft_A, lf.fft_B}) {
+            const FftPlan &q = p->ffts[f];
+            std::fprintf(stderr, "  plan %d: M %d stages %d logC %d tw_off %d tw_count %d radices", f, q.M, q.nstages, q.logC, q.tw_off, q.tw_count);
+            for (int j = 0; j < q.nstages; ++j) std::fprintf(stderr, " %d(s%d)", q.radix[j], q.stride[j]);
+            std::fprintf(stderr, "\n");
+        }
+        for (int c = 0; c < kNumClasses; ++c)
+            std::fprintf(stderr, "  class %d: bands %d threads %d items %d max_elems %d\n", c, p->cls[c].n_bands, p->cls[c].threads,
+                         p->cls[c].items_per_cta, p->cls[c].max_elems);
+    }
     if (p->device < 0) { *out = p; return CQT_OK; }
 
     // ---- device tables
     int cur = 0;
     if (cudaGetDevice(&cur) != cudaSuccess || cudaSetDevice(p->device) != cudaSuccess) { p->device = -1; delete p; return CQT_ERR_CUDA; }
     std::vector<float> tA(L.table_len), tS(L.table_len), tTA(L.table_len), tSA(L.table_len);
-    std::vector<int2> span(L.bands.size());
     for (size_t i = 0; i < L.bands.size(); ++i) {
         const HostBand &hb = L.bands[i];
-        span[i] = make_int2((int)(hb.kc + hb.d0 + hb.j_lo), (int)hb.y_off);
         for (int64_t j = 0; j < hb.S; ++j) {
             const int64_t k = hb.kc + hb.d0 + j;
             const double g = L.g[hb.tab_off + j], h = L.h[hb.tab_off + j];
@@ -295,7 +317,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     chk(upload(p->d.tab_analysis_adj, tTA));
     chk(upload(p->d.tab_synthesis_adj, tSA));
     chk(upload(p->d.cover, cover));
-    chk(upload(p->d.span, span));
+    chk(upload(p->d.dbg, std::vector<int>(8, 0)));
     for (auto &c : p->cls) chk(upload(c.d_work, c.work));
     cudaDeviceProp prop;
     chk(cudaGetDeviceProperties(&prop, p->device));
@@ -349,7 +371,16 @@ cqt_status cqt_plan_tables(const cqt_plan *p, const float **g_host, const float 
     return CQT_OK;
 }
 
-cqt_status cqt_plan_check(const cqt_plan *p) { return p ? CQT_OK : CQT_ERR_INVALID_ARG; }
+cqt_status cqt_plan_check(const cqt_plan *p) {
+    if (!p) return CQT_ERR_INVALID_ARG;
+    if (p->device < 0 || !p->d.dbg) return CQT_OK;
+    int w[8];
+    if (cudaMemcpy(w, p->d.dbg, sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess) return CQT_ERR_CUDA;
+    if (w[0] == 0) return CQT_OK;
+    std::fprintf(stderr, "cqt debug check: site %d index %lld limit %lld block (%d,%d) thread %d\n", w[0],
+                 ((long long)w[2] << 32) | (unsigned)w[1], ((long long)w[4] << 32) | (unsigned)w[3], w[5], w[6], w[7]);
+    return CQT_ERR_DEVICE_CHECK;
+}
 
 }  // extern "C"
 

@@ -30,6 +30,8 @@ struct BandArgs {
     long long coeff_count;
     float2 *Y;               // synthesis form: weighted-bin rows
     long long y_pitch;
+    long long table_len;
+    int *dbg;
 };
 
 // THREADS / MINB: launch bounds of the class (64 registers per thread when THREADS * MINB = 1024 ... 2048)
@@ -65,8 +67,10 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
         if (m <= last_pos) d = m;
         else if (m >= first_neg) d = m - M;
         else return make_float2(0.f, 0.f);
+        if (!CQT_CHK(a.dbg, 301, br.tab_off + (d - br.d0), a.table_len)) return make_float2(0.f, 0.f);
         const float g = __ldg(tab + (d - br.d0));
         const int k = br.kc + d;
+        if (!CQT_CHK(a.dbg, 302, k < 0 ? -k : (k > half ? a.N - k : k), half + 1)) return make_float2(0.f, 0.f);
         float2 xv;
         if (k < 0) xv = cconj(__ldg(X + (-k)));
         else if (k > half) xv = cconj(__ldg(X + (a.N - k)));
@@ -84,8 +88,8 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     }
     float2 *tws = buf + M + 16;
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
-    const Tile t{buf, 1, 1, 0u};
-    auto store = [&](int n, int, float2 v) { out[n] = v; };
+    const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
+    auto store = [&](int n, int, float2 v) { if (CQT_CHK(a.dbg, 303, n, M)) out[n] = v; };
     fft_fused<+1, Sync, false, true, false, true, false>(t, fp, tws, load, store, tid, nthr);
 }
 
@@ -105,6 +109,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     // adjoint of analysis, sidebands: U[m] + conj U[-m] is the DFT of 2 Re c
     const bool fold = a.fold && br.side != 0;
     auto load = [&](int n, int) -> float2 {
+        if (!CQT_CHK(a.dbg, 304, n, M)) return make_float2(0.f, 0.f);
         float2 v = __ldg(in + n);
         if (fold) v = make_float2(2.f * v.x, 0.f);
         return v;
@@ -112,16 +117,18 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     const float *tab = a.table + br.tab_off;
     float2 *Y = a.Y + (long long)ch * a.y_pitch + br.y_off;
     const int last_pos = br.d0 + br.S - 1, first_neg = M + br.d0;
-    // slot m -> offset d -> support index j -> entry j - j_lo of the band's weighted-bin run
+    // slot m -> offset d -> bin kc + d of the band's plane (only bins 0..N/2 are kept)
+    const int half = a.N >> 1;
     auto store = [&](int m, int, float2 u) {
         int d;
         if (m <= last_pos) d = m;
         else if (m >= first_neg) d = m - M;
         else return;
-        const int j = d - br.d0, i = j - br.j_lo;
-        if (i < 0 || i >= br.n_in) return;
-        const float h = __ldg(tab + j);
-        Y[i] = make_float2(h * u.x, h * u.y);
+        const int k = br.kc + d;
+        if (k < 0 || k > half) return;
+        if (!CQT_CHK(a.dbg, 305, br.tab_off + (d - br.d0), a.table_len)) return;
+        const float h = __ldg(tab + (d - br.d0));
+        if (CQT_CHK(a.dbg, 306, (long long)br.y_off + k, a.y_pitch)) Y[k] = make_float2(h * u.x, h * u.y);
     };
     if (fp.generic) {
         float2 *alt = buf + M;
@@ -133,7 +140,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     }
     float2 *tws = buf + M + 16;
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
-    const Tile t{buf, 1, 1, 0u};
+    const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
     fft_fused<-1, Sync, false, true, false, true, false>(t, fp, tws, load, store, tid, nthr);
 }
 
@@ -150,6 +157,8 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
     a.max_elems = c.max_elems;
     a.coeff_count = p.lay.coeff_count;
     a.y_pitch = p.y_pitch;
+    a.table_len = p.lay.table_len;
+    a.dbg = p.d.dbg;
     return a;
 }
 

@@ -124,11 +124,11 @@ __global__ void __launch_bounds__(512) huge_rows_kernel(HugeArgs a) {
             if (m <= last_pos) d = (int)m;
             else if (m >= first_neg) d = (int)(m - M);
             else continue;
-            const int j = d - a.br.d0, i = j - a.br.j_lo;
-            if (i < 0 || i >= a.br.n_in) continue;
+            const int k = a.br.kc + d;
+            if (k < 0 || k > (a.N >> 1)) continue;
             const float2 u = buf[(size_t)dif_pos(fp, q) * pitch + r];
-            const float h = __ldg(tab + j);
-            Y[i] = make_float2(h * u.x, h * u.y);
+            const float h = __ldg(tab + (d - a.br.d0));
+            Y[k] = make_float2(h * u.x, h * u.y);
         }
     }
 }

@@ -139,7 +139,7 @@ __device__ void fft_dif(float2 *buf, float2 *alt, int pitch, int ncols, uint32_t
         break;
         if (POW2) {
             switch (r) {
-                CQT_STAGE(2) CQT_STAGE(4) CQT_STAGE(8) CQT_STAGE(16) CQT_STAGE(32)
+                CQT_STAGE(2) CQT_STAGE(4) CQT_STAGE(8) CQT_STAGE(16)
                 default: break;
             }
         } else {
@@ -178,16 +178,24 @@ __device__ __forceinline__ float2 twiddle_s(const float2 *tw, int logC, uint32_t
     return cmul(tw[y & (C - 1)], tw[C + (y >> logC)]);
 }
 
-template <int R>
-__device__ __forceinline__ void apply_twiddle_powers(float2 w1, float (&re)[R], float (&im)[R]) {
+// Multiplies re/im[q] by w^q, q = 1 .. R-1, where w = exp(-+2 pi i y1 / M).  The powers w^1, w^2, w^4, w^8
+// are looked up (two-level table), the others are products of at most three of those: raising one rounded
+// w to the q-th power would multiply its phase error by q, a product of looked-up factors only adds errors.
+template <int R, int SIGN>
+__device__ __forceinline__ void apply_twiddle_powers(const float2 *tw, int logC, uint32_t y1, float (&re)[R], float (&im)[R]) {
     float wr[R], wi[R];
     wr[0] = 1.f; wi[0] = 0.f;
-    wr[1] = w1.x; wi[1] = w1.y;
 #pragma unroll
-    for (int q = 2; q < R; ++q) {
-        const int a = (q + 1) / 2, b = q / 2;
-        wr[q] = fmaf(wr[a], wr[b], -wi[a] * wi[b]);
-        wi[q] = fmaf(wr[a], wi[b], wi[a] * wr[b]);
+    for (int q = 1; q < R; ++q) {
+        if ((q & (q - 1)) == 0) {
+            const float2 w = twiddle_s(tw, logC, y1 * q);
+            wr[q] = w.x;
+            wi[q] = SIGN > 0 ? -w.y : w.y;
+        } else {
+            const int hb = q >= 8 ? 8 : (q >= 4 ? 4 : 2), lo = q - hb;
+            wr[q] = fmaf(wr[hb], wr[lo], -wi[hb] * wi[lo]);
+            wi[q] = fmaf(wr[hb], wi[lo], wi[hb] * wr[lo]);
+        }
     }
 #pragma unroll
     for (int q = 1; q < R; ++q) {
@@ -202,7 +210,25 @@ struct Tile {
     int pitch;             // elements between consecutive positions
     int ncols;             // interleaved columns
     uint32_t ncols_magic;
+    int limit;             // elements available at buf (checked in CQT_DEBUG_BOUNDS builds)
+    int *dbg;              // debug status words (may be null)
 };
+
+// Debug build (-DCQT_DEBUG_BOUNDS): every instrumented access checks its index, records the first
+// violation {site, index, limit, block x, block y, thread} in the plan's status words and skips the access.
+#ifdef CQT_DEBUG_BOUNDS
+__device__ __forceinline__ bool dbg_ok(int *dbg, int site, long long idx, long long limit) {
+    if (idx >= 0 && idx < limit) return true;
+    if (dbg && atomicCAS(&dbg[0], 0, site) == 0) {
+        dbg[1] = (int)idx; dbg[2] = (int)(idx >> 32); dbg[3] = (int)limit; dbg[4] = (int)(limit >> 32);
+        dbg[5] = blockIdx.x; dbg[6] = blockIdx.y; dbg[7] = threadIdx.x;
+    }
+    return false;
+}
+#define CQT_CHK(dbg, site, idx, limit) cqt::dbg_ok(dbg, site, (long long)(idx), (long long)(limit))
+#else
+#define CQT_CHK(dbg, site, idx, limit) true
+#endif
 
 // first stage: operands from load(pos, col); results to shared memory.
 // COLFAST: consecutive threads take consecutive columns, else consecutive butterflies.
@@ -233,12 +259,12 @@ __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, co
         }
         if (base == 0) Sync::sync();
         if (active) {
-            float2 w1 = twiddle_s(tw, fp.logC, b);
-            if (SIGN > 0) w1.y = -w1.y;
-            apply_twiddle_powers<R>(w1, re, im);
+            apply_twiddle_powers<R, SIGN>(tw, fp.logC, b, re, im);
             float2 *p = t.buf + (size_t)b * t.pitch + col;
 #pragma unroll
-            for (int q = 0; q < R; ++q) p[(size_t)q * spad * t.pitch] = make_float2(re[q], im[q]);
+            for (int q = 0; q < R; ++q)
+                if (CQT_CHK(t.dbg, 101, (size_t)b * t.pitch + col + (size_t)q * spad * t.pitch, t.limit))
+                    p[(size_t)q * spad * t.pitch] = make_float2(re[q], im[q]);
         }
     }
 }
@@ -258,15 +284,14 @@ __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, c
         float2 *p = t.buf + (size_t)pos * t.pitch + col;
         const int step = s * t.pitch;
         float re[R], im[R];
+        if (!CQT_CHK(t.dbg, 102, (size_t)pos * t.pitch + col + (size_t)(R - 1) * step, t.limit)) continue;
 #pragma unroll
         for (int q = 0; q < R; ++q) {
             const float2 v = p[q * step];
             re[q] = v.x; im[q] = v.y;
         }
         if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
-        float2 w1 = twiddle_s(tw, fp.logC, np * tmul);
-        if (SIGN > 0) w1.y = -w1.y;
-        apply_twiddle_powers<R>(w1, re, im);
+        apply_twiddle_powers<R, SIGN>(tw, fp.logC, np * tmul, re, im);
 #pragma unroll
         for (int q = 0; q < R; ++q) p[q * step] = make_float2(re[q], im[q]);
     }
@@ -313,6 +338,7 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
         if (PAD) pos += fp.pad_delta ? fastdiv(b, fp.k1magic[d - 1], fp.k1div[d - 1]) : 0u;
         const float2 *p = t.buf + (size_t)pos * t.pitch + col;
         float re[R], im[R];
+        if (!CQT_CHK(t.dbg, 103, (size_t)pos * t.pitch + col + (size_t)(R - 1) * t.pitch, t.limit)) continue;
 #pragma unroll
         for (int q = 0; q < R; ++q) {
             const float2 v = p[q * t.pitch];
@@ -341,7 +367,7 @@ __device__ __forceinline__ void only_stage(const Tile &t, Load load, Store store
 }
 
 #define CQT_RADIX_CASES_ALL(X) X(2) X(3) X(4) X(5) X(6) X(8) X(9) X(10) X(12) X(15) X(16)
-#define CQT_RADIX_CASES_POW2(X) X(2) X(4) X(8) X(16) X(32)
+#define CQT_RADIX_CASES_POW2(X) X(2) X(4) X(8) X(16)
 
 // Runs the first `nrun` stages of the plan (nrun = nstages: the whole transform with the last stage fused
 // into `store`; nrun = nstages - 1... not offered: use fft_fused_keep for "results stay in shared memory").
@@ -352,6 +378,7 @@ template <int SIGN, class Sync, bool POW2, bool PAD, bool COLFAST_IN, bool REV, 
 __device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, Store store, int tid, int nthr) {
     const int d = fp.nstages;
     if (d == 1) {
+        Sync::sync();   // tables staged by the caller become visible to the functors
 #define X(RR) case RR: only_stage<RR, SIGN>(t, load, store, tid, nthr); break;
         if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
         else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }

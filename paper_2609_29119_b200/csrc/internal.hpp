@@ -28,7 +28,9 @@ struct LongFft {
     int fft_A = -1, fft_B = -1;   // FftPlan indices
     int tw_lp = 0, tw_n = 0;      // two-level tables of W_Lp and W_N inside the twiddle array
     int log_lp_c = 0, log_n_c = 0;
-    int tw_rows = 1;              // rows per mirrored half handled by one CTA of the row kernels
+    int n_lp = 0, n_n = 0;        // entry counts of those tables
+    int tw_rows = 1;              // rows per mirrored half handled by one CTA of the forward row kernel
+    int tw_rows_inv = 1;          // rows per CTA of the inverse row kernel
     int tw_cols = 1;              // columns per CTA of the column kernels
     int64_t x_pitch = 0;          // elements per signal of the half-spectrum buffer (Lp + 1 rounded up)
 };
@@ -51,7 +53,7 @@ struct DevicePlan {
     float *tab_analysis_adj = nullptr; // N g / (2 M)
     float *tab_synthesis_adj = nullptr;// h w_k / N
     int32_t *cover = nullptr;          // per bin: (first covering band << 8) | count
-    int2 *span = nullptr;              // per band: (first in-range bin, offset in the weighted-bin row)
+    int *dbg = nullptr;                // 8 status words of the debug-bounds build
 };
 
 }  // namespace cqt
@@ -63,7 +65,9 @@ struct cqt_plan {
     std::vector<cqt::BandRec> bands;
     int device = -1;
     int64_t N = 0;
-    int64_t y_pitch = 0;
+    int64_t y_pitch = 0;               // weighted-bin scratch elements per signal (y_planes * y_plane)
+    int64_t y_plane = 0;               // elements per plane (N/2 + 1 rounded up)
+    int y_planes = 1;                  // largest number of bands covering one bin
     cqt::LongFft lf;
     cqt::BandClass cls[cqt::kNumClasses];
     std::vector<cqt::HugeBand> huge;

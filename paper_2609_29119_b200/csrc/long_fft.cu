@@ -5,7 +5,8 @@
 //
 // Index split:  sample index j = j1 * B + j2,  bin index k = k1 + A * k2  (j1,k1 < A; j2,k2 < B).
 //   forward  pass C ("columns"): for TWc adjacent j2, A-point DFT over j1, times W_Lp^{j2 k1},
-//                                written to T[k1][j2].
+//                                written to T[k1][j2].  First stage on registers straight from the
+//                                signal (packing on load), last stage straight to T.
 //            pass R ("rows"):    for a set of rows k1, B-point DFT over j2 gives Z[k1 + A k2];
 //                                a CTA owns TWr rows and their mirror images A - k1 (plus one
 //                                extra row each side) so both operands of Eq. untangle are in its
@@ -15,6 +16,10 @@
 //                                written to T[q1][j2].
 //            pass C':            inverse A-point DFT over q1, scaled, unpacked to x[2j], x[2j+1].
 // When Lp is small (A == 1) the row kernels read / write the signal directly and passes C, C' vanish.
+//
+// Weighted-bin scratch: P planes of Lp+1 bins per signal; band b writes plane b mod P, where P is the
+// largest number of bands covering one bin, so two bands of one plane never share a bin and the sum
+// over the bands covering bin k reads planes (lo + i) mod P, i < n, at index k: coalesced, no atomics.
 #include "engine.cuh"
 #include "internal.hpp"
 
@@ -27,8 +32,8 @@ struct LongArgs {
     const float2 *tw;
     int fft_A, fft_B;
     int A, B, Lp;
-    int tw_lp, log_lp_c;   // two-level table of W_Lp
-    int tw_n, log_n_c;     // two-level table of W_N
+    int tw_lp, log_lp_c, n_lp;   // two-level table of W_Lp and its entry count
+    int tw_n, log_n_c, n_n;      // two-level table of W_N
     int tw_cols, tw_rows;
     int valid_len;
     int aligned;           // signal rows allow float2 access
@@ -41,11 +46,13 @@ struct LongArgs {
     long long x_pitch;
     // inverse gather
     const float2 *Y;
-    long long y_pitch;
+    long long y_pitch;     // per signal
+    long long y_plane;     // per plane
+    int planes;
     const int32_t *cover;
-    const int2 *span;
     float scale;
-    uint32_t cols_magic, rows_magic;
+    uint32_t cols_magic, rows_magic, planes_magic;
+    int *dbg;
 };
 
 __device__ __forceinline__ float2 load_packed(const float *row, long long j, int valid_len, int aligned) {
@@ -68,33 +75,36 @@ __device__ __forceinline__ void store_packed(float *row, long long j, float2 v, 
     }
 }
 
+__device__ __forceinline__ void stage_table(float2 *dst, const float2 *__restrict__ src, int n, int tid, int nthr) {
+    for (int i = tid; i < n; i += nthr) dst[i] = __ldg(src + i);
+}
+
 // ---------------------------------------------------------------- forward, pass C
-__global__ void __launch_bounds__(512) rfft_cols_fwd_kernel(LongArgs a) {
+__global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
     const int j2_0 = blockIdx.x * TW;
     const int ch = blockIdx.y;
     const FftPlan &fp = a.ffts[a.fft_A];
     float2 *buf = smem_long;
+    float2 *tws = buf + (size_t)a.A * TW;
+    float2 *wl = tws + fp.tw_count;
+    stage_twiddles(tws, a.tw, fp, tid, nthr);
+    stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
     const float *row = a.x_in + (long long)ch * a.x_stride;
-    const int total = a.A * TW;
-    for (int e = tid; e < total; e += nthr) {
-        const int j1 = e / TW, c = e - j1 * TW;
-        buf[e] = load_packed(row, (long long)j1 * a.B + j2_0 + c, a.valid_len, a.aligned);
-    }
-    __syncthreads();
-    fft_dif<-1, BlockSync, true>(buf, nullptr, TW, TW, a.cols_magic, fp, a.tw, tid, nthr);
     float2 *T = a.T + (long long)ch * a.t_pitch;
-    const float2 *wl = a.tw + a.tw_lp;
-    for (int e = tid; e < total; e += nthr) {
-        const int k1 = e / TW, c = e - k1 * TW;
-        const float2 v = buf[dif_pos(fp, k1) * TW + c];
-        const float2 w = twiddle(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
-        T[(long long)k1 * a.B + j2_0 + c] = cmul(v, w);
-    }
+    const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
+    auto load = [&](int j1, int c) -> float2 {
+        return load_packed(row, (long long)j1 * a.B + j2_0 + c, a.valid_len, a.aligned);
+    };
+    auto store = [&](int k1, int c, float2 v) {
+        const float2 w = twiddle_s(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
+        if (CQT_CHK(a.dbg, 201, (long long)k1 * a.B + j2_0 + c, a.Lp)) T[(long long)k1 * a.B + j2_0 + c] = cmul(v, w);
+    };
+    fft_fused<-1, BlockSync, true, false, true, false, true>(t, fp, tws, load, store, tid, nthr);
 }
 
-// rows owned by CTA t of the row kernels: first set TWr*t + i, second set A - TWr*t - TWr + i
+// rows owned by CTA t of the forward row kernel: first set TWr*t + i, second set A - TWr*t - TWr + i
 // (i < TWr owned; i == TWr is the extra, read-only row of each set; row A means row 0)
 __device__ __forceinline__ int row_of(int t, int r, int TW, int A) {
     const int i = r <= TW ? r : r - (TW + 1);
@@ -103,29 +113,33 @@ __device__ __forceinline__ int row_of(int t, int r, int TW, int A) {
 }
 
 // ---------------------------------------------------------------- forward, pass R (+ untangle)
-__global__ void __launch_bounds__(512) rfft_rows_fwd_kernel(LongArgs a) {
+__global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
     const int A = a.A, B = a.B, TW = a.tw_rows;
     const bool direct = (A == 1);
     const int ncols = direct ? 1 : 2 * TW + 2;
-    const int pitch = direct ? 1 : ncols + 1;   // odd: the transposing load is conflict-free
+    const int pitch = direct ? 1 : ncols + 1;   // odd: the transposing accesses are conflict-free
     const FftPlan &fp = a.ffts[a.fft_B];
     float2 *buf = smem_long;
+    float2 *tws = buf + (size_t)B * pitch;
+    float2 *wn = tws + fp.tw_count;
+    stage_twiddles(tws, a.tw, fp, tid, nthr);
+    stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
+    const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
     if (direct) {
         const float *row = a.x_in + (long long)ch * a.x_stride;
-        for (int e = tid; e < B; e += nthr) buf[e] = load_packed(row, e, a.valid_len, a.aligned);
+        auto load = [&](int j, int) -> float2 { return load_packed(row, j, a.valid_len, a.aligned); };
+        fft_fused_keep<-1, BlockSync, true, false>(tile, fp, tws, load, tid, nthr);
     } else {
         const float2 *T = a.T + (long long)ch * a.t_pitch;
-        for (int e = tid; e < ncols * B; e += nthr) {
-            const int r = e / B, j2 = e - r * B;
-            buf[(size_t)j2 * pitch + r] = __ldg(T + (long long)row_of(t, r, TW, A) * B + j2);
-        }
+        auto load = [&](int j2, int r) -> float2 {
+            const long long i = (long long)row_of(t, r, TW, A) * B + j2;
+            return CQT_CHK(a.dbg, 202, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
+        };
+        fft_fused_keep<-1, BlockSync, true, false>(tile, fp, tws, load, tid, nthr);
     }
-    __syncthreads();
-    fft_dif<-1, BlockSync, true>(buf, nullptr, pitch, ncols, a.rows_magic, fp, a.tw, tid, nthr);
     float2 *X = a.X + (long long)ch * a.x_pitch;
-    const float2 *wn = a.tw + a.tw_n;
     const int nown = direct ? 1 : 2 * TW;
     for (int e = tid; e < nown * B; e += nthr) {
         const int k2 = e / nown, o = e - k2 * nown;
@@ -141,11 +155,14 @@ __global__ void __launch_bounds__(512) rfft_rows_fwd_kernel(LongArgs a) {
         }
         const int k1 = direct ? 0 : row_of(t, r, TW, A);
         if (!direct && k1 == 0) { rp = r; k2p = k2 == 0 ? 0 : B - k2; }
+        const int k = k1 + A * k2;
+        if (!CQT_CHK(a.dbg, 203, k, a.Lp) || !CQT_CHK(a.dbg, 204, (size_t)dif_pos(fp, k2p) * pitch + rp, B * pitch) ||
+            !CQT_CHK(a.dbg, 209, (size_t)dif_pos(fp, k2) * pitch + r, B * pitch))
+            continue;
         const float2 z = buf[(size_t)dif_pos(fp, k2) * pitch + r];
         const float2 zp = buf[(size_t)dif_pos(fp, k2p) * pitch + rp];
-        const int k = k1 + A * k2;
         // X_k = 1/2 (1 - i w) Z_k + 1/2 (1 + i w) conj Z_{Lp-k},  w = exp(-2 pi i k / N)
-        const float2 w = twiddle(wn, a.log_n_c, (uint32_t)k);
+        const float2 w = twiddle_s(wn, a.log_n_c, (uint32_t)k);
         const float2 ev = make_float2(0.5f * (z.x + zp.x), 0.5f * (z.y - zp.y));   // (Z + conj Zp)/2
         const float2 od = make_float2(0.5f * (z.x - zp.x), 0.5f * (z.y + zp.y));   // (Z - conj Zp)/2
         // -i w od = (w.y od.x + w.x od.y) + i (w.y od.y - w.x od.x)
@@ -156,21 +173,24 @@ __global__ void __launch_bounds__(512) rfft_rows_fwd_kernel(LongArgs a) {
 }
 
 // ---------------------------------------------------------------- inverse, pass R' (gather + retangle)
-__device__ __forceinline__ float2 gather_bin(const float2 *__restrict__ Y, const int32_t *__restrict__ cover,
-                                             const int2 *__restrict__ span, int k) {
-    const int32_t cv = __ldg(cover + k);
+// sum over the bands covering bin k, in band order
+__device__ __forceinline__ float2 gather_bin(const LongArgs &a, const float2 *__restrict__ Y, int k) {
+    if (!CQT_CHK(a.dbg, 205, k, a.Lp + 1)) return make_float2(0.f, 0.f);
+    const int32_t cv = __ldg(a.cover + k);
     const int lo = cv >> 8, n = cv & 255;
+    if (!CQT_CHK(a.dbg, 206, n, a.planes + 1)) return make_float2(0.f, 0.f);
+    int plane = lo - (int)fastdiv(lo, a.planes_magic, a.planes) * a.planes;
     float2 acc = make_float2(0.f, 0.f);
     for (int i = 0; i < n; ++i) {
-        const int2 sp = __ldg(span + lo + i);
-        const float2 v = __ldg(Y + sp.y + (k - sp.x));
+        const float2 v = __ldg(Y + (long long)plane * a.y_plane + k);
         acc.x += v.x;
         acc.y += v.y;
+        if (++plane == a.planes) plane = 0;
     }
     return acc;
 }
 
-__global__ void __launch_bounds__(512) irfft_rows_kernel(LongArgs a) {
+__global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
     const int A = a.A, B = a.B, TW = a.tw_rows, Lp = a.Lp;
@@ -179,63 +199,65 @@ __global__ void __launch_bounds__(512) irfft_rows_kernel(LongArgs a) {
     const int pitch = direct ? 1 : (TW | 1);
     const FftPlan &fp = a.ffts[a.fft_B];
     float2 *buf = smem_long;
+    float2 *tws = buf + (size_t)B * pitch;
+    float2 *wn = tws + fp.tw_count;
+    float2 *wl = wn + a.n_n;
+    stage_twiddles(tws, a.tw, fp, tid, nthr);
+    stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
+    if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
+    __syncthreads();   // the operand functor below reads the W_N table
     const float2 *Y = a.Y + (long long)ch * a.y_pitch;
-    const float2 *wn = a.tw + a.tw_n;
-    for (int e = tid; e < ncols * B; e += nthr) {
-        const int q2 = e / ncols, r = e - q2 * ncols;
+    const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
+    auto load = [&](int q2, int r) -> float2 {
         const int q1 = direct ? 0 : t * TW + r;
         const int q = q1 + A * q2;
-        float2 xq = gather_bin(Y, a.cover, a.span, q);
-        float2 xm = gather_bin(Y, a.cover, a.span, Lp - q);
+        float2 xq = gather_bin(a, Y, q);
+        float2 xm = gather_bin(a, Y, Lp - q);
         if (q == 0) { xq.y = 0.f; xm.y = 0.f; }   // bins 0 and N/2 are made real
         // Z_q = 1/2 [(1 + i conj w) X_q + (1 - i conj w) conj X_{Lp-q}],  w = exp(-2 pi i q / N)
-        const float2 w = twiddle(wn, a.log_n_c, (uint32_t)q);
+        const float2 w = twiddle_s(wn, a.log_n_c, (uint32_t)q);
         const float2 ev = make_float2(xq.x + xm.x, xq.y - xm.y);   // X_q + conj X_m
         const float2 od = make_float2(xq.x - xm.x, xq.y + xm.y);   // X_q - conj X_m
-        // i conj(w) od = i (w.x - i w.y)... conj w = (w.x, -w.y); i*conj w = (w.y, w.x)
-        const float2 icw = make_float2(w.y, w.x);
-        const float2 rot = cmul(icw, od);
-        buf[(size_t)q2 * pitch + r] = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
-    }
-    __syncthreads();
-    fft_dif<+1, BlockSync, true>(buf, nullptr, pitch, ncols, a.rows_magic, fp, a.tw, tid, nthr);
+        const float2 rot = cmul(make_float2(w.y, w.x), od);        // i conj(w) = (w.y, w.x)
+        return make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
+    };
+    fft_fused_keep<+1, BlockSync, true, true>(tile, fp, tws, load, tid, nthr);
     if (direct) {
         float *row = a.x_out + (long long)ch * a.x_stride;
         for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[dif_pos(fp, j)], a.valid_len, a.aligned);
     } else {
         float2 *T = a.T + (long long)ch * a.t_pitch;
-        const float2 *wl = a.tw + a.tw_lp;
         for (int e = tid; e < ncols * B; e += nthr) {
             const int r = e / B, j2 = e - r * B;
             const int q1 = t * TW + r;
             const float2 v = buf[(size_t)dif_pos(fp, j2) * pitch + r];
-            const float2 w = cconj(twiddle(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
-            T[(long long)q1 * B + j2] = cmul(v, w);
+            const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
+            if (CQT_CHK(a.dbg, 207, (long long)q1 * B + j2, a.Lp)) T[(long long)q1 * B + j2] = cmul(v, w);
         }
     }
 }
 
 // ---------------------------------------------------------------- inverse, pass C' (+ unpack)
-__global__ void __launch_bounds__(512) irfft_cols_kernel(LongArgs a) {
+__global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
     const int j2_0 = blockIdx.x * TW;
     const int ch = blockIdx.y;
     const FftPlan &fp = a.ffts[a.fft_A];
     float2 *buf = smem_long;
+    float2 *tws = buf + (size_t)a.A * TW;
+    stage_twiddles(tws, a.tw, fp, tid, nthr);
     const float2 *T = a.T + (long long)ch * a.t_pitch;
-    const int total = a.A * TW;
-    for (int e = tid; e < total; e += nthr) {
-        const int q1 = e / TW, c = e - q1 * TW;
-        buf[e] = __ldg(T + (long long)q1 * a.B + j2_0 + c);
-    }
-    __syncthreads();
-    fft_dif<+1, BlockSync, true>(buf, nullptr, TW, TW, a.cols_magic, fp, a.tw, tid, nthr);
     float *row = a.x_out + (long long)ch * a.x_stride;
-    for (int e = tid; e < total; e += nthr) {
-        const int j1 = e / TW, c = e - j1 * TW;
-        store_packed(row, (long long)j1 * a.B + j2_0 + c, buf[dif_pos(fp, j1) * TW + c], a.valid_len, a.aligned);
-    }
+    const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
+    auto load = [&](int q1, int c) -> float2 {
+        const long long i = (long long)q1 * a.B + j2_0 + c;
+        return CQT_CHK(a.dbg, 208, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
+    };
+    auto store = [&](int j1, int c, float2 v) {
+        store_packed(row, (long long)j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned);
+    };
+    fft_fused<+1, BlockSync, true, false, true, false, true>(t, fp, tws, load, store, tid, nthr);
 }
 
 // ---------------------------------------------------------------- host side
@@ -252,8 +274,10 @@ static LongArgs base_args(const cqt_plan &p, int64_t valid_len, int64_t x_stride
     a.Lp = (int)p.lf.Lp;
     a.tw_lp = p.lf.tw_lp;
     a.log_lp_c = p.lf.log_lp_c;
+    a.n_lp = p.lf.n_lp;
     a.tw_n = p.lf.tw_n;
     a.log_n_c = p.lf.log_n_c;
+    a.n_n = p.lf.n_n;
     a.tw_cols = p.lf.tw_cols;
     a.tw_rows = p.lf.tw_rows;
     a.valid_len = (int)valid_len;
@@ -262,19 +286,31 @@ static LongArgs base_args(const cqt_plan &p, int64_t valid_len, int64_t x_stride
     a.t_pitch = p.lf.Lp;
     a.x_pitch = p.lf.x_pitch;
     a.y_pitch = p.y_pitch;
+    a.y_plane = p.y_plane;
+    a.planes = p.y_planes;
+    a.planes_magic = magic_of(p.y_planes);
     a.cover = p.d.cover;
-    a.span = p.d.span;
     a.cols_magic = magic_of(a.tw_cols);
+    a.dbg = p.d.dbg;
     return a;
 }
 
-static size_t rows_fwd_smem(const LongFft &lf) {
-    return lf.A == 1 ? (size_t)lf.B * 8 : (size_t)lf.B * (2 * lf.tw_rows + 3) * 8;
+static size_t plan_tw(const cqt_plan &p, int fft) { return (size_t)p.ffts[fft].tw_count; }
+
+static size_t rows_fwd_smem(const cqt_plan &p) {
+    const LongFft &lf = p.lf;
+    const size_t data = lf.A == 1 ? (size_t)lf.B : (size_t)lf.B * (2 * lf.tw_rows + 3);
+    return (data + plan_tw(p, lf.fft_B) + lf.n_n) * 8;
 }
-static size_t rows_inv_smem(const LongFft &lf) {
-    return lf.A == 1 ? (size_t)lf.B * 8 : (size_t)lf.B * (lf.tw_rows | 1) * 8;
+static size_t rows_inv_smem(const cqt_plan &p) {
+    const LongFft &lf = p.lf;
+    const size_t data = lf.A == 1 ? (size_t)lf.B : (size_t)lf.B * (lf.tw_rows_inv | 1);
+    return (data + plan_tw(p, lf.fft_B) + lf.n_n + (lf.A == 1 ? 0 : lf.n_lp)) * 8;
 }
-static size_t cols_smem(const LongFft &lf) { return (size_t)lf.A * lf.tw_cols * 8; }
+static size_t cols_smem(const cqt_plan &p) {
+    const LongFft &lf = p.lf;
+    return ((size_t)lf.A * lf.tw_cols + plan_tw(p, lf.fft_A) + lf.n_lp) * 8;
+}
 
 static int threads_for(size_t butterflies) {
     int t = 64;
@@ -291,17 +327,17 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
     const LongFft &lf = p.lf;
     if (lf.A > 1) {
         dim3 grid((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
-        rfft_cols_fwd_kernel<<<grid, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(lf), st>>>(a);
+        rfft_cols_fwd_kernel<<<grid, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), st>>>(a);
         note_launch(p, "rfft_cols_fwd", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         a.rows_magic = magic_of(2 * lf.tw_rows + 2);
         dim3 grid2((unsigned)(lf.A / (2 * lf.tw_rows)), (unsigned)batch);
-        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows + 2) / 8), rows_fwd_smem(lf), st>>>(a);
+        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows + 2) / 8), rows_fwd_smem(p), st>>>(a);
     } else {
         a.rows_magic = 0;
         dim3 grid2(1, (unsigned)batch);
-        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B / 8), rows_fwd_smem(lf), st>>>(a);
+        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B / 8), rows_fwd_smem(p), st>>>(a);
     }
     note_launch(p, "rfft_rows_fwd", st);
     return cudaGetLastError();
@@ -316,19 +352,20 @@ cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, f
     a.scale = (float)(0.5 / (double)p.lf.Lp);
     const LongFft &lf = p.lf;
     if (lf.A > 1) {
-        a.rows_magic = magic_of(lf.tw_rows);
-        dim3 grid((unsigned)(lf.A / lf.tw_rows), (unsigned)batch);
-        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B * lf.tw_rows / 8), rows_inv_smem(lf), st>>>(a);
+        a.rows_magic = magic_of(lf.tw_rows_inv);
+        a.tw_rows = lf.tw_rows_inv;
+        dim3 grid((unsigned)(lf.A / lf.tw_rows_inv), (unsigned)batch);
+        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B * lf.tw_rows_inv / 8), rows_inv_smem(p), st>>>(a);
         note_launch(p, "irfft_rows", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         dim3 grid2((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
-        irfft_cols_kernel<<<grid2, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(lf), st>>>(a);
+        irfft_cols_kernel<<<grid2, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), st>>>(a);
         note_launch(p, "irfft_cols", st);
     } else {
         a.rows_magic = 0;
         dim3 grid(1, (unsigned)batch);
-        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B / 8), rows_inv_smem(lf), st>>>(a);
+        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B / 8), rows_inv_smem(p), st>>>(a);
         note_launch(p, "irfft_rows", st);
     }
     return cudaGetLastError();
@@ -336,14 +373,14 @@ cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, f
 
 cudaError_t configure_long_fft_kernels(const cqt_plan &p) {
     cudaError_t e;
-    e = cudaFuncSetAttribute(rfft_rows_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_fwd_smem(p.lf));
+    e = cudaFuncSetAttribute(rfft_rows_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_fwd_smem(p));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(irfft_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_inv_smem(p.lf));
+    e = cudaFuncSetAttribute(irfft_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_inv_smem(p));
     if (e != cudaSuccess) return e;
     if (p.lf.A > 1) {
-        e = cudaFuncSetAttribute(rfft_cols_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p.lf));
+        e = cudaFuncSetAttribute(rfft_cols_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(irfft_cols_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p.lf));
+        e = cudaFuncSetAttribute(irfft_cols_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
     }
     return e;
 }

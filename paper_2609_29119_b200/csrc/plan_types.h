@@ -37,7 +37,7 @@ struct BandRec {
     int32_t M;          // coefficients
     int32_t tab_off;    // into the window tables (S entries, offset order)
     int32_t coeff_off;  // into one signal's coefficient row
-    int32_t y_off;      // into one signal's weighted-bin scratch row (in-range entries only)
+    int32_t y_off;      // offset of the band's plane in one signal's weighted-bin scratch (entries indexed by bin)
     int32_t j_lo;       // first support index whose bin lies in 0..N/2
     int32_t n_in;       // number of support entries whose bin lies in 0..N/2
     int32_t side;       // 0 regular, 1 DC, 2 Nyquist
