@@ -94,7 +94,7 @@ void note_launch(const cqt_plan &p, const char *name, cudaStream_t st);
 // long_fft.cu
 cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,
                                 float2 *T, float2 *X, cudaStream_t st);
-cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, float *x, int64_t x_stride,
+cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, float2 *T, float *x, int64_t x_stride,
                                 int64_t batch, int64_t valid_len, cudaStream_t st);
 cudaError_t configure_long_fft_kernels(const cqt_plan &p);
 

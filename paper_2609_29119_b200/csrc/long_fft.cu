@@ -45,6 +45,8 @@ struct LongArgs {
     float2 *X;             // half spectrum rows (forward)
     long long x_pitch;
     // inverse gather
+    float2 *Z;             // packed spectrum rows assembled by the gather kernel (inverse)
+    int log_b, log_own;    // log2 B, log2 (2 TWr)
     const float2 *Y;
     long long y_pitch;     // per signal
     long long y_plane;     // per plane
@@ -142,7 +144,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     float2 *X = a.X + (long long)ch * a.x_pitch;
     const int nown = direct ? 1 : 2 * TW;
     for (int e = tid; e < nown * B; e += nthr) {
-        const int k2 = e / nown, o = e - k2 * nown;
+        const int k2 = direct ? e : e >> a.log_own, o = e - k2 * nown;
         // owned row o -> column index r in shared memory, and the partner's column / k2
         int r, rp, k2p;
         if (direct) {
@@ -172,7 +174,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     }
 }
 
-// ---------------------------------------------------------------- inverse, pass R' (gather + retangle)
+// ---------------------------------------------------------------- inverse: overlap-add + retangle
 // sum over the bands covering bin k, in band order
 __device__ __forceinline__ float2 gather_bin(const LongArgs &a, const float2 *__restrict__ Y, int k) {
     if (!CQT_CHK(a.dbg, 205, k, a.Lp + 1)) return make_float2(0.f, 0.f);
@@ -190,36 +192,55 @@ __device__ __forceinline__ float2 gather_bin(const LongArgs &a, const float2 *__
     return acc;
 }
 
+// One thread per pair (q, Lp - q), 0 <= q <= Lp/2: every bin of the half spectrum is summed once, both
+// packed bins of the pair follow from the same two values (Eq. retangle with w_{Lp-q} = -conj w_q):
+//   Z_q      = s [ (X_q + conj X_m) + i conj(w) (X_q - conj X_m) ]
+//   Z_{Lp-q} = s [ (X_m + conj X_q) - i w (X_m - conj X_q) ],   m = Lp - q, w = exp(-2 pi i q / N), s = 1/(2 Lp)
+__global__ void __launch_bounds__(256) gather_retangle_kernel(LongArgs a) {
+    const int ch = blockIdx.y;
+    const int Lp = a.Lp;
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q > (Lp >> 1)) return;
+    const float2 *Y = a.Y + (long long)ch * a.y_pitch;
+    float2 *Z = a.Z + (long long)ch * a.t_pitch;
+    const int m = Lp - q;
+    float2 xq = gather_bin(a, Y, q);
+    float2 xm = gather_bin(a, Y, m);
+    if (q == 0) { xq.y = 0.f; xm.y = 0.f; }   // bins 0 and N/2 are made real
+    const float2 w = twiddle(a.tw + a.tw_n, a.log_n_c, (uint32_t)q);
+    {
+        const float2 ev = make_float2(xq.x + xm.x, xq.y - xm.y);   // X_q + conj X_m
+        const float2 od = make_float2(xq.x - xm.x, xq.y + xm.y);   // X_q - conj X_m
+        const float2 rot = cmul(make_float2(w.y, w.x), od);        // i conj(w) = (w.y, w.x)
+        Z[q] = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
+    }
+    if (q != 0 && m != q) {
+        const float2 ev = make_float2(xm.x + xq.x, xm.y - xq.y);   // X_m + conj X_q
+        const float2 od = make_float2(xm.x - xq.x, xm.y + xq.y);   // X_m - conj X_q
+        const float2 rot = cmul(make_float2(w.y, -w.x), od);       // -i w = (w.y, -w.x)
+        Z[m] = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
+    }
+}
+
+// ---------------------------------------------------------------- inverse, pass R'
 __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
-    const int A = a.A, B = a.B, TW = a.tw_rows, Lp = a.Lp;
+    const int A = a.A, B = a.B, TW = a.tw_rows;
     const bool direct = (A == 1);
     const int ncols = direct ? 1 : TW;
     const int pitch = direct ? 1 : (TW | 1);
     const FftPlan &fp = a.ffts[a.fft_B];
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)B * pitch;
-    float2 *wn = tws + fp.tw_count;
-    float2 *wl = wn + a.n_n;
+    float2 *wl = tws + fp.tw_count;
     stage_twiddles(tws, a.tw, fp, tid, nthr);
-    stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
     if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
-    __syncthreads();   // the operand functor below reads the W_N table
-    const float2 *Y = a.Y + (long long)ch * a.y_pitch;
+    const float2 *Z = a.Z + (long long)ch * a.t_pitch;
     const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
     auto load = [&](int q2, int r) -> float2 {
-        const int q1 = direct ? 0 : t * TW + r;
-        const int q = q1 + A * q2;
-        float2 xq = gather_bin(a, Y, q);
-        float2 xm = gather_bin(a, Y, Lp - q);
-        if (q == 0) { xq.y = 0.f; xm.y = 0.f; }   // bins 0 and N/2 are made real
-        // Z_q = 1/2 [(1 + i conj w) X_q + (1 - i conj w) conj X_{Lp-q}],  w = exp(-2 pi i q / N)
-        const float2 w = twiddle_s(wn, a.log_n_c, (uint32_t)q);
-        const float2 ev = make_float2(xq.x + xm.x, xq.y - xm.y);   // X_q + conj X_m
-        const float2 od = make_float2(xq.x - xm.x, xq.y + xm.y);   // X_q - conj X_m
-        const float2 rot = cmul(make_float2(w.y, w.x), od);        // i conj(w) = (w.y, w.x)
-        return make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
+        const long long i = (long long)(direct ? 0 : t * TW + r) + (long long)A * q2;
+        return CQT_CHK(a.dbg, 210, i, a.Lp) ? __ldg(Z + i) : make_float2(0.f, 0.f);
     };
     fft_fused_keep<+1, BlockSync, true, true>(tile, fp, tws, load, tid, nthr);
     if (direct) {
@@ -228,7 +249,7 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     } else {
         float2 *T = a.T + (long long)ch * a.t_pitch;
         for (int e = tid; e < ncols * B; e += nthr) {
-            const int r = e / B, j2 = e - r * B;
+            const int r = e >> a.log_b, j2 = e - (r << a.log_b);
             const int q1 = t * TW + r;
             const float2 v = buf[(size_t)dif_pos(fp, j2) * pitch + r];
             const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
@@ -292,6 +313,10 @@ static LongArgs base_args(const cqt_plan &p, int64_t valid_len, int64_t x_stride
     a.cover = p.d.cover;
     a.cols_magic = magic_of(a.tw_cols);
     a.dbg = p.d.dbg;
+    a.log_b = 0;
+    while ((1ll << a.log_b) < p.lf.B) ++a.log_b;
+    a.log_own = 0;
+    while ((1 << a.log_own) < 2 * p.lf.tw_rows) ++a.log_own;
     return a;
 }
 
@@ -305,7 +330,7 @@ static size_t rows_fwd_smem(const cqt_plan &p) {
 static size_t rows_inv_smem(const cqt_plan &p) {
     const LongFft &lf = p.lf;
     const size_t data = lf.A == 1 ? (size_t)lf.B : (size_t)lf.B * (lf.tw_rows_inv | 1);
-    return (data + plan_tw(p, lf.fft_B) + lf.n_n + (lf.A == 1 ? 0 : lf.n_lp)) * 8;
+    return (data + plan_tw(p, lf.fft_B) + (lf.A == 1 ? 0 : lf.n_lp)) * 8;
 }
 static size_t cols_smem(const cqt_plan &p) {
     const LongFft &lf = p.lf;
@@ -343,14 +368,22 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
     return cudaGetLastError();
 }
 
-cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, float *x, int64_t x_stride,
+cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, float2 *T, float *x, int64_t x_stride,
                                 int64_t batch, int64_t valid_len, cudaStream_t st) {
     LongArgs a = base_args(p, valid_len, x_stride, x);
     a.x_out = x;
     a.T = T;
+    a.Z = Z;
     a.Y = Y;
     a.scale = (float)(0.5 / (double)p.lf.Lp);
     const LongFft &lf = p.lf;
+    {
+        dim3 grid((unsigned)((lf.Lp / 2 + 1 + 255) / 256), (unsigned)batch);
+        gather_retangle_kernel<<<grid, 256, 0, st>>>(a);
+        note_launch(p, "gather_retangle", st);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     if (lf.A > 1) {
         a.rows_magic = magic_of(lf.tw_rows_inv);
         a.tw_rows = lf.tw_rows_inv;
