@@ -165,7 +165,7 @@ def kernel_algorithmic_bytes(plan, w, batch):
         cls_m[bi.launch_class] = cls_m.get(bi.launch_class, 0) + bi.M
         cls_s[bi.launch_class] = cls_s.get(bi.launch_class, 0) + bi.support
     sig = 4 * w.valid_len * batch
-    two_pass = plan.N // 2 > 16384
+    two_pass = plan.N // 2 > 4096
     out = {"rfft_cols_fwd": sig if two_pass else 0, "rfft_rows_fwd": 0 if two_pass else sig,
            "irfft_cols": sig if two_pass else 0, "irfft_rows": 0 if two_pass else sig}
     for c in cls_m:

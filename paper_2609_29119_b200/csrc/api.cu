@@ -95,6 +95,19 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp) {
     fp.logC = logC;
     fp.tw_count = (int32_t)((1ll << logC) + (M + (1ll << logC) - 1) / (1ll << logC));
     fp.pad_delta = (fp.nstages > 1 && (fp.stride[0] % 2 == 0)) ? 1 : 0;
+    fp.tw_full_off = -1;
+    if (pow2) {
+        fp.tw_full_off = (int32_t)tw.size();
+        for (int64_t y = 0; y < M; ++y) {
+            const double ang = -2.0 * kPi * (double)y / (double)M;
+            tw.push_back(make_float2((float)std::cos(ang), (float)std::sin(ang)));
+        }
+        for (int j = 0; j < fp.nstages; ++j) {
+            int l = 0;
+            while ((1 << l) < fp.radix[j]) ++l;
+            fp.lg[j] = l;
+        }
+    }
     return true;
 }
 
@@ -118,6 +131,11 @@ void free_device(cqt_plan *p) {
     cudaFree(p->d.cover); cudaFree(p->d.dbg);
     for (auto &c : p->cls) cudaFree(c.d_work);
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
+    for (int i = 0; i < 2; ++i) {
+        if (p->aux[i]) cudaStreamDestroy(p->aux[i]);
+        if (p->ev_join[i]) cudaEventDestroy(p->ev_join[i]);
+    }
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     cudaSetDevice(cur);
 }
 
@@ -189,7 +207,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     };
     LongFft &lf = p->lf;
     lf.Lp = N / 2;
-    if (lf.Lp <= 16384) { lf.A = 1; lf.B = lf.Lp; }
+    if (lf.Lp <= 4096) { lf.A = 1; lf.B = lf.Lp; }   // one CTA per signal: data and full twiddle table in shared memory
     else {
         int lg = 0;
         while ((1ll << lg) < lf.Lp) ++lg;
@@ -323,6 +341,11 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     chk(cudaGetDeviceProperties(&prop, p->device));
     p->sm_count = prop.multiProcessorCount;
     p->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+        chk(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
+        chk(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
+    }
+    chk(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
     if (e == cudaSuccess) chk(configure_band_kernels(*p));
     if (e == cudaSuccess) chk(configure_long_fft_kernels(*p));
     if (e == cudaSuccess) chk(configure_huge_kernels(*p));

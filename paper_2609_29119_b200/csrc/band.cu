@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
     const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
     auto store = [&](int n, int, float2 v) { if (CQT_CHK(a.dbg, 303, n, M)) out[n] = v; };
-    fft_fused<+1, Sync, false, true, false, true, false>(t, fp, tws, load, store, tid, nthr);
+    fft_fused<+1, Sync, false, true, false, true, false, false>(t, fp, tws, load, store, tid, nthr);
 }
 
 template <int THREADS, int MINB, bool WARP>
@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     float2 *tws = buf + M + 16;
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
     const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
-    fft_fused<-1, Sync, false, true, false, true, false>(t, fp, tws, load, store, tid, nthr);
+    fft_fused<-1, Sync, false, true, false, true, false, false>(t, fp, tws, load, store, tid, nthr);
 }
 
 static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *table, int64_t batch) {
@@ -187,8 +187,32 @@ static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, Ba
     return e;
 }
 
+// The classes of one call are independent (disjoint outputs), and the short-band classes alone leave most SMs
+// idle, so they run on two helper streams beside the long-band classes: fork after the caller's stream, join
+// back into it.  With event timing on, everything stays on the caller's stream.
+struct ForkJoin {
+    const cqt_plan &p;
+    cudaStream_t st;
+    bool used[2] = {false, false};
+    bool serial;
+    ForkJoin(const cqt_plan &plan, cudaStream_t s) : p(plan), st(s), serial(plan.timing || !plan.aux[0] || !plan.aux[1]) {
+        if (!serial) cudaEventRecord(p.ev_fork, st);
+    }
+    cudaStream_t stream_for(int cls) {
+        if (serial || cls >= 3 || p.cls[cls].n_bands == 0) return st;
+        const int i = cls == 2 ? 0 : 1;
+        if (!used[i]) { cudaStreamWaitEvent(p.aux[i], p.ev_fork, 0); used[i] = true; }
+        return p.aux[i];
+    }
+    void join() {
+        for (int i = 0; i < 2; ++i)
+            if (used[i]) { cudaEventRecord(p.ev_join[i], p.aux[i]); cudaStreamWaitEvent(st, p.ev_join[i], 0); }
+    }
+};
+
 cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
                                        int64_t batch, cudaStream_t st) {
+    ForkJoin fj(p, st);
     static const char *names[kNumClasses] = {"bands_from_spectrum/class0", "bands_from_spectrum/class1",
                                               "bands_from_spectrum/class2", "bands_from_spectrum/class3",
                                               "bands_from_spectrum/class4"};
@@ -197,14 +221,16 @@ cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, co
         a.spec = X;
         a.spec_pitch = p.lf.x_pitch;
         a.coef = c;
-        cudaError_t e = launch_class<true>(p, i, names[i], a, st);
-        if (e != cudaSuccess) return e;
+        cudaError_t e = launch_class<true>(p, i, names[i], a, fj.stream_for(i));
+        if (e != cudaSuccess) { fj.join(); return e; }
     }
+    fj.join();
     return cudaSuccess;
 }
 
 cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool fold_sidebands, const float2 *c,
                                      float2 *Y, int64_t batch, cudaStream_t st) {
+    ForkJoin fj(p, st);
     static const char *names[kNumClasses] = {"bands_to_spectrum/class0", "bands_to_spectrum/class1",
                                               "bands_to_spectrum/class2", "bands_to_spectrum/class3",
                                               "bands_to_spectrum/class4"};
@@ -213,9 +239,10 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
         a.coef = const_cast<float2 *>(c);
         a.Y = Y;
         a.fold = fold_sidebands ? 1 : 0;
-        cudaError_t e = launch_class<false>(p, i, names[i], a, st);
-        if (e != cudaSuccess) return e;
+        cudaError_t e = launch_class<false>(p, i, names[i], a, fj.stream_for(i));
+        if (e != cudaSuccess) { fj.join(); return e; }
     }
+    fj.join();
     return cudaSuccess;
 }
 

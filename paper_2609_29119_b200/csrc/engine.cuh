@@ -205,6 +205,31 @@ __device__ __forceinline__ void apply_twiddle_powers(const float2 *tw, int logC,
     }
 }
 
+// Same with a full table twf[y] = exp(-2 pi i y / M): one load per power, no products (short power-of-two plans).
+template <int R, int SIGN>
+__device__ __forceinline__ void apply_twiddle_direct(const float2 *twf, uint32_t y1, float (&re)[R], float (&im)[R]) {
+#pragma unroll
+    for (int q = 1; q < R; ++q) {
+        const float2 w = twf[y1 * q];
+        const float wi = SIGN > 0 ? -w.y : w.y;
+        const float x = re[q], y = im[q];
+        re[q] = fmaf(x, w.x, -y * wi);
+        im[q] = fmaf(x, wi, y * w.x);
+    }
+}
+
+// position of frequency k for a power-of-two plan: digit reversal by shifts
+__device__ __forceinline__ uint32_t dif_pos_pow2(const FftPlan &fp, uint32_t k) {
+    uint32_t pos = 0, rem = k;
+#pragma unroll 1
+    for (int j = 0; j < fp.nstages; ++j) {
+        const int l = fp.lg[j];
+        pos = (pos << l) | (rem & ((1u << l) - 1));
+        rem >>= l;
+    }
+    return pos;
+}
+
 struct Tile {
     float2 *buf;
     int pitch;             // elements between consecutive positions
@@ -232,7 +257,7 @@ __device__ __forceinline__ bool dbg_ok(int *dbg, int site, long long idx, long l
 
 // first stage: operands from load(pos, col); results to shared memory.
 // COLFAST: consecutive threads take consecutive columns, else consecutive butterflies.
-template <int R, int SIGN, bool PAD, bool COLFAST, class Sync, class Load>
+template <int R, int SIGN, bool PAD, bool COLFAST, bool DIRECT, class Sync, class Load>
 __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
     const int s = fp.stride[0];
     const int total = s * t.ncols;
@@ -259,7 +284,8 @@ __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, co
         }
         if (base == 0) Sync::sync();
         if (active) {
-            apply_twiddle_powers<R, SIGN>(tw, fp.logC, b, re, im);
+            if (DIRECT) apply_twiddle_direct<R, SIGN>(tw, b, re, im);
+            else apply_twiddle_powers<R, SIGN>(tw, fp.logC, b, re, im);
             float2 *p = t.buf + (size_t)b * t.pitch + col;
 #pragma unroll
             for (int q = 0; q < R; ++q)
@@ -269,7 +295,7 @@ __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, co
     }
 }
 
-template <int R, int SIGN, bool PAD>
+template <int R, int SIGN, bool PAD, bool DIRECT>
 __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, const float2 *tw, int j, int n_cur, int tmul,
                                              int tid, int nthr) {
     const int s = fp.stride[j];
@@ -291,7 +317,8 @@ __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, c
             re[q] = v.x; im[q] = v.y;
         }
         if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
-        apply_twiddle_powers<R, SIGN>(tw, fp.logC, np * tmul, re, im);
+        if (DIRECT) { if (s > 1) apply_twiddle_direct<R, SIGN>(tw, np * tmul, re, im); }
+        else apply_twiddle_powers<R, SIGN>(tw, fp.logC, np * tmul, re, im);
 #pragma unroll
         for (int q = 0; q < R; ++q) p[q * step] = make_float2(re[q], im[q]);
     }
@@ -374,7 +401,7 @@ __device__ __forceinline__ void only_stage(const Tile &t, Load load, Store store
 // Requires a non-generic plan.  tw = shared-memory copy of the plan's two-level table, written by the
 // caller (stage_twiddles) WITHOUT a barrier after it: the first stage synchronises once its operand loads
 // are issued.  The routine synchronises between stages, not at the end.
-template <int SIGN, class Sync, bool POW2, bool PAD, bool COLFAST_IN, bool REV, bool COLFAST_OUT, class Load, class Store>
+template <int SIGN, class Sync, bool POW2, bool PAD, bool COLFAST_IN, bool REV, bool COLFAST_OUT, bool DIRECT, class Load, class Store>
 __device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, Store store, int tid, int nthr) {
     const int d = fp.nstages;
     if (d == 1) {
@@ -385,7 +412,7 @@ __device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Lo
 #undef X
         return;
     }
-#define X(RR) case RR: first_stage<RR, SIGN, PAD, COLFAST_IN, Sync>(t, fp, tw, load, tid, nthr); break;
+#define X(RR) case RR: first_stage<RR, SIGN, PAD, COLFAST_IN, DIRECT, Sync>(t, fp, tw, load, tid, nthr); break;
     if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
     else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
@@ -393,7 +420,7 @@ __device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Lo
     int n_cur = fp.stride[0], tmul = fp.radix[0];
 #pragma unroll 1
     for (int j = 1; j < d - 1; ++j) {
-#define X(RR) case RR: middle_stage<RR, SIGN, PAD>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+#define X(RR) case RR: middle_stage<RR, SIGN, PAD, DIRECT>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
         if (POW2) { switch (fp.radix[j]) { CQT_RADIX_CASES_POW2(X) default: break; } }
         else { switch (fp.radix[j]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
@@ -409,7 +436,7 @@ __device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Lo
 
 // Same, but every stage after the first runs in shared memory and the results stay there
 // (digit-reversed positions, see dif_pos); ends with a sync.
-template <int SIGN, class Sync, bool POW2, bool COLFAST_IN, class Load>
+template <int SIGN, class Sync, bool POW2, bool COLFAST_IN, bool DIRECT, class Load>
 __device__ void fft_fused_keep(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
     const int d = fp.nstages;
     if (d == 1) {
@@ -421,7 +448,7 @@ __device__ void fft_fused_keep(const Tile &t, const FftPlan &fp, const float2 *t
         Sync::sync();
         return;
     }
-#define X(RR) case RR: first_stage<RR, SIGN, false, COLFAST_IN, Sync>(t, fp, tw, load, tid, nthr); break;
+#define X(RR) case RR: first_stage<RR, SIGN, false, COLFAST_IN, DIRECT, Sync>(t, fp, tw, load, tid, nthr); break;
     if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
     else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
@@ -429,7 +456,7 @@ __device__ void fft_fused_keep(const Tile &t, const FftPlan &fp, const float2 *t
     int n_cur = fp.stride[0], tmul = fp.radix[0];
 #pragma unroll 1
     for (int j = 1; j < d; ++j) {
-#define X(RR) case RR: middle_stage<RR, SIGN, false>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+#define X(RR) case RR: middle_stage<RR, SIGN, false, DIRECT>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
         if (POW2) { switch (fp.radix[j]) { CQT_RADIX_CASES_POW2(X) default: break; } }
         else { switch (fp.radix[j]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X

@@ -77,6 +77,12 @@ __device__ __forceinline__ void store_packed(float *row, long long j, float2 v, 
     }
 }
 
+// copies the full twiddle table of a power-of-two plan into shared memory
+__device__ __forceinline__ void stage_full(float2 *dst, const float2 *__restrict__ tw_base, const FftPlan &fp, int tid, int nthr) {
+    const float2 *src = tw_base + fp.tw_full_off;
+    for (int i = tid; i < fp.M; i += nthr) dst[i] = __ldg(src + i);
+}
+
 __device__ __forceinline__ void stage_table(float2 *dst, const float2 *__restrict__ src, int n, int tid, int nthr) {
     for (int i = tid; i < n; i += nthr) dst[i] = __ldg(src + i);
 }
@@ -90,8 +96,8 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     const FftPlan &fp = a.ffts[a.fft_A];
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)a.A * TW;
-    float2 *wl = tws + fp.tw_count;
-    stage_twiddles(tws, a.tw, fp, tid, nthr);
+    float2 *wl = tws + fp.M;
+    stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
     const float *row = a.x_in + (long long)ch * a.x_stride;
     float2 *T = a.T + (long long)ch * a.t_pitch;
@@ -103,7 +109,7 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
         const float2 w = twiddle_s(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
         if (CQT_CHK(a.dbg, 201, (long long)k1 * a.B + j2_0 + c, a.Lp)) T[(long long)k1 * a.B + j2_0 + c] = cmul(v, w);
     };
-    fft_fused<-1, BlockSync, true, false, true, false, true>(t, fp, tws, load, store, tid, nthr);
+    fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
 }
 
 // rows owned by CTA t of the forward row kernel: first set TWr*t + i, second set A - TWr*t - TWr + i
@@ -125,44 +131,47 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     const FftPlan &fp = a.ffts[a.fft_B];
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)B * pitch;
-    float2 *wn = tws + fp.tw_count;
-    stage_twiddles(tws, a.tw, fp, tid, nthr);
+    float2 *wn = tws + fp.M;
+    stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
     const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
     if (direct) {
         const float *row = a.x_in + (long long)ch * a.x_stride;
         auto load = [&](int j, int) -> float2 { return load_packed(row, j, a.valid_len, a.aligned); };
-        fft_fused_keep<-1, BlockSync, true, false>(tile, fp, tws, load, tid, nthr);
+        fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
     } else {
         const float2 *T = a.T + (long long)ch * a.t_pitch;
         auto load = [&](int j2, int r) -> float2 {
             const long long i = (long long)row_of(t, r, TW, A) * B + j2;
             return CQT_CHK(a.dbg, 202, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
         };
-        fft_fused_keep<-1, BlockSync, true, false>(tile, fp, tws, load, tid, nthr);
+        fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
     }
     float2 *X = a.X + (long long)ch * a.x_pitch;
+    // epilogue: each thread keeps one owned row (column o) and walks k2; for rows other than k1 = 0 the partner
+    // Z_{Lp-k} sits in the mirror row at k2' = B-1-k2, whose position is the digit-wise complement B-1-pos(k2)
     const int nown = direct ? 1 : 2 * TW;
-    for (int e = tid; e < nown * B; e += nthr) {
-        const int k2 = direct ? e : e >> a.log_own, o = e - k2 * nown;
-        // owned row o -> column index r in shared memory, and the partner's column / k2
-        int r, rp, k2p;
-        if (direct) {
-            r = 0; rp = 0; k2p = k2 == 0 ? 0 : B - k2;
-        } else {
-            r = o < TW ? o : o + 1;                      // skip the extra row of the first set
-            const int i = o < TW ? o : o - TW;
-            rp = o < TW ? (TW + 1) + (TW - i) : (TW - i);   // mirror row's column
-            k2p = B - 1 - k2;
-        }
-        const int k1 = direct ? 0 : row_of(t, r, TW, A);
-        if (!direct && k1 == 0) { rp = r; k2p = k2 == 0 ? 0 : B - k2; }
+    const int o = direct ? 0 : (tid & (nown - 1));
+    const int kstart = direct ? tid : (tid >> a.log_own), kstep = direct ? nthr : (nthr >> a.log_own);
+    int r = 0, rp = 0;
+    if (!direct) {
+        r = o < TW ? o : o + 1;                          // skip the extra row of the first set
+        const int i = o < TW ? o : o - TW;
+        rp = o < TW ? (TW + 1) + (TW - i) : (TW - i);    // mirror row's column
+    }
+    const int k1 = direct ? 0 : row_of(t, r, TW, A);
+    for (int k2 = kstart; k2 < B; k2 += kstep) {
+        const uint32_t pos = dif_pos_pow2(fp, k2);
+        uint32_t posp;
+        int rpp = rp;
+        if (k1 == 0) { rpp = r; posp = k2 == 0 ? 0u : dif_pos_pow2(fp, B - k2); }
+        else posp = (uint32_t)(B - 1) - pos;
         const int k = k1 + A * k2;
-        if (!CQT_CHK(a.dbg, 203, k, a.Lp) || !CQT_CHK(a.dbg, 204, (size_t)dif_pos(fp, k2p) * pitch + rp, B * pitch) ||
-            !CQT_CHK(a.dbg, 209, (size_t)dif_pos(fp, k2) * pitch + r, B * pitch))
+        if (!CQT_CHK(a.dbg, 203, k, a.Lp) || !CQT_CHK(a.dbg, 204, (size_t)posp * pitch + rpp, B * pitch) ||
+            !CQT_CHK(a.dbg, 209, (size_t)pos * pitch + r, B * pitch))
             continue;
-        const float2 z = buf[(size_t)dif_pos(fp, k2) * pitch + r];
-        const float2 zp = buf[(size_t)dif_pos(fp, k2p) * pitch + rp];
+        const float2 z = buf[(size_t)pos * pitch + r];
+        const float2 zp = buf[(size_t)posp * pitch + rpp];
         // X_k = 1/2 (1 - i w) Z_k + 1/2 (1 + i w) conj Z_{Lp-k},  w = exp(-2 pi i k / N)
         const float2 w = twiddle_s(wn, a.log_n_c, (uint32_t)k);
         const float2 ev = make_float2(0.5f * (z.x + zp.x), 0.5f * (z.y - zp.y));   // (Z + conj Zp)/2
@@ -233,8 +242,8 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     const FftPlan &fp = a.ffts[a.fft_B];
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)B * pitch;
-    float2 *wl = tws + fp.tw_count;
-    stage_twiddles(tws, a.tw, fp, tid, nthr);
+    float2 *wl = tws + fp.M;
+    stage_full(tws, a.tw, fp, tid, nthr);
     if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
     const float2 *Z = a.Z + (long long)ch * a.t_pitch;
     const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
@@ -242,16 +251,16 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
         const long long i = (long long)(direct ? 0 : t * TW + r) + (long long)A * q2;
         return CQT_CHK(a.dbg, 210, i, a.Lp) ? __ldg(Z + i) : make_float2(0.f, 0.f);
     };
-    fft_fused_keep<+1, BlockSync, true, true>(tile, fp, tws, load, tid, nthr);
+    fft_fused_keep<+1, BlockSync, true, true, true>(tile, fp, tws, load, tid, nthr);
     if (direct) {
         float *row = a.x_out + (long long)ch * a.x_stride;
-        for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[dif_pos(fp, j)], a.valid_len, a.aligned);
+        for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[dif_pos_pow2(fp, j)], a.valid_len, a.aligned);
     } else {
         float2 *T = a.T + (long long)ch * a.t_pitch;
         for (int e = tid; e < ncols * B; e += nthr) {
             const int r = e >> a.log_b, j2 = e - (r << a.log_b);
             const int q1 = t * TW + r;
-            const float2 v = buf[(size_t)dif_pos(fp, j2) * pitch + r];
+            const float2 v = buf[(size_t)dif_pos_pow2(fp, j2) * pitch + r];
             const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
             if (CQT_CHK(a.dbg, 207, (long long)q1 * B + j2, a.Lp)) T[(long long)q1 * B + j2] = cmul(v, w);
         }
@@ -267,7 +276,7 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     const FftPlan &fp = a.ffts[a.fft_A];
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)a.A * TW;
-    stage_twiddles(tws, a.tw, fp, tid, nthr);
+    stage_full(tws, a.tw, fp, tid, nthr);
     const float2 *T = a.T + (long long)ch * a.t_pitch;
     float *row = a.x_out + (long long)ch * a.x_stride;
     const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
@@ -278,7 +287,7 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     auto store = [&](int j1, int c, float2 v) {
         store_packed(row, (long long)j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned);
     };
-    fft_fused<+1, BlockSync, true, false, true, false, true>(t, fp, tws, load, store, tid, nthr);
+    fft_fused<+1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
 }
 
 // ---------------------------------------------------------------- host side
@@ -320,7 +329,7 @@ static LongArgs base_args(const cqt_plan &p, int64_t valid_len, int64_t x_stride
     return a;
 }
 
-static size_t plan_tw(const cqt_plan &p, int fft) { return (size_t)p.ffts[fft].tw_count; }
+static size_t plan_tw(const cqt_plan &p, int fft) { return (size_t)p.ffts[fft].M; }
 
 static size_t rows_fwd_smem(const cqt_plan &p) {
     const LongFft &lf = p.lf;

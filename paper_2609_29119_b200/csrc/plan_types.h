@@ -20,13 +20,14 @@ struct FftPlan {
     int32_t generic;                // 1 if stage 0 is a generic (out-of-place) radix
     int32_t tw_count;               // entries of the two-level table (C + ceil(M / C))
     int32_t pad_delta;              // 1 if single-column buffers skip one element per s_0 positions (bank spread)
-    int32_t pad_[1];
+    int32_t tw_full_off;            // power-of-two plans: offset of the full table exp(-2 pi i y / M), y < M; else -1
     int32_t radix[kMaxStages];
     int32_t stride[kMaxStages];     // s_j
     uint32_t rmagic[kMaxStages];    // ceil(2^32 / r_j)
     uint32_t smagic[kMaxStages];    // ceil(2^32 / s_j)
     int32_t k1div[kMaxStages];      // s_0 / n_j: butterfly blocks of stage j per first-stage output digit
     uint32_t k1magic[kMaxStages];
+    int32_t lg[kMaxStages];         // log2 r_j for power-of-two plans
 };
 
 // One band of the layout as the kernels see it.
