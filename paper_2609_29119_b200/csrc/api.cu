@@ -40,6 +40,13 @@ const int kBandRadices[] = {16, 15, 12, 10, 9, 8, 6, 5, 4, 3, 2};
 const int kPow2Radices[] = {16, 8, 4, 2};
 
 // fewest stages, then smallest largest radix
+int g_radix_cap = 16;   // set around the planning of two-pass sub-transforms
+int max_band_radix() {
+    int cap = g_radix_cap;
+    if (const char *v = std::getenv("CQT_MAX_RADIX")) { const int r = std::atoi(v); if (r >= 5) cap = std::min(cap, r); }
+    return cap;
+}
+
 bool best_split(int64_t m, const int *radices, int nr, std::map<int64_t, std::vector<int>> &memo, std::vector<int> &out) {
     if (m == 1) { out.clear(); return true; }
     auto it = memo.find(m);
@@ -47,7 +54,7 @@ bool best_split(int64_t m, const int *radices, int nr, std::map<int64_t, std::ve
     std::vector<int> best;
     for (int i = 0; i < nr; ++i) {
         const int r = radices[i];
-        if (m % r) continue;
+        if (m % r || r > max_band_radix()) continue;
         std::vector<int> sub;
         if (!best_split(m / r, radices, nr, memo, sub)) continue;
         sub.push_back(r);
@@ -60,7 +67,7 @@ bool best_split(int64_t m, const int *radices, int nr, std::map<int64_t, std::ve
 }
 
 // returns false if M cannot be planned
-bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp) {
+bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp, bool want_full = false) {
     std::memset(&fp, 0, sizeof(fp));
     fp.M = (int32_t)M;
     int64_t smooth = M, rest = 1;
@@ -96,13 +103,13 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp) {
     fp.tw_count = (int32_t)((1ll << logC) + (M + (1ll << logC) - 1) / (1ll << logC));
     fp.pad_delta = (fp.nstages > 1 && (fp.stride[0] % 2 == 0)) ? 1 : 0;
     fp.tw_full_off = -1;
-    if (pow2) {
+    if (pow2 || want_full) {
         fp.tw_full_off = (int32_t)tw.size();
         for (int64_t y = 0; y < M; ++y) {
             const double ang = -2.0 * kPi * (double)y / (double)M;
             tw.push_back(make_float2((float)std::cos(ang), (float)std::sin(ang)));
         }
-        for (int j = 0; j < fp.nstages; ++j) {
+        for (int j = 0; j < fp.nstages && pow2; ++j) {
             int l = 0;
             while ((1 << l) < fp.radix[j]) ++l;
             fp.lg[j] = l;
@@ -130,6 +137,7 @@ void free_device(cqt_plan *p) {
     cudaFree(p->d.tab_analysis_adj); cudaFree(p->d.tab_synthesis_adj);
     cudaFree(p->d.cover); cudaFree(p->d.dbg);
     for (auto &c : p->cls) cudaFree(c.d_work);
+    for (auto &g : p->two_pass) cudaFree(g.d_recs);
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     for (int i = 0; i < 2; ++i) {
         if (p->aux[i]) cudaStreamDestroy(p->aux[i]);
@@ -196,12 +204,12 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     // ---- transform-length plans and twiddles
     std::vector<float2> tw;
     std::map<int64_t, int> fft_of;
-    auto plan_for = [&](int64_t M, bool pow2) -> int {
-        const int64_t key = pow2 ? -M : M;
+    auto plan_for = [&](int64_t M, bool pow2, bool full = false) -> int {
+        const int64_t key = pow2 ? -M : (full ? M + (1ll << 40) : M);
         auto it = fft_of.find(key);
         if (it != fft_of.end()) return it->second;
         FftPlan fp;
-        if (!make_fft_plan(M, pow2, tw, fp)) return -1;
+        if (!make_fft_plan(M, pow2, tw, fp, full)) return -1;
         p->ffts.push_back(fp);
         return fft_of[key] = (int)p->ffts.size() - 1;
     };
@@ -236,16 +244,21 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         br.y_off = (int32_t)((int64_t)(i % p->y_planes) * p->y_plane);
         br.j_lo = (int32_t)hb.j_lo; br.n_in = (int32_t)hb.n_in; br.side = hb.side;
         br.inv_M = (float)(1.0 / (double)hb.M);
-        br.fft = plan_for(hb.M, false);
-        if (br.fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
+        br.fft = -1;
     }
     // ---- launch classes by band length
     // class 0: one warp per item, 8 items per CTA; the others one CTA per item, sized so that several CTAs
     // share an SM (64 registers per thread) except for the longest bands, which fill its shared memory
-    const int limits[kNumClasses] = {128, 1024, 4096, 13500, 1 << 30};
-    const int threads[kNumClasses] = {256, 64, 256, 512, 1024};
+    int limits[kNumClasses] = {128, 1024, 4096, 13500, 1 << 30};
+    int threads[kNumClasses] = {256, 64, 256, 512, 1024};
+    int minb[kNumClasses] = {2, 16, 4, 2, 1};
+    // tuning hooks (experiments): CQT_CLASSk="limit,threads,min_blocks", CQT_MAX_RADIX=r
     for (int c = 0; c < kNumClasses; ++c) {
+        char name[32];
+        std::snprintf(name, sizeof(name), "CQT_CLASS%d", c);
+        if (const char *v = std::getenv(name)) std::sscanf(v, "%d,%d,%d", &limits[c], &threads[c], &minb[c]);
         p->cls[c].threads = threads[c];
+        p->cls[c].min_blocks = minb[c];
         p->cls[c].items_per_cta = c == 0 ? 8 : 1;
     }
     std::vector<int> order(L.bands.size());
@@ -257,38 +270,76 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         const long long v = std::atoll(cap);
         if (v >= 64 && v < smem_cap_elems) smem_cap_elems = v;
     }
+    // bands above this length take the two-pass kernels (small tiles, many CTAs per SM)
+    int64_t two_pass_min = 1ll << 40;   // by default only bands too long for one CTA's shared memory
+    if (const char *v = std::getenv("CQT_TWO_PASS_MIN")) two_pass_min = std::max<long long>(64, std::atoll(v));
+    // M = A * B with plannable factors: fewest stages, then the most balanced split; 0 if there is none
+    int tp_radix_cap = 16;
+    if (const char *v = std::getenv("CQT_TP_MAX_RADIX")) tp_radix_cap = std::max(5, std::atoi(v));
+    auto split_two_pass = [&](int64_t M) -> int64_t {
+        g_radix_cap = tp_radix_cap;
+        int64_t bestA = 0;
+        int best_cost = 1 << 30;
+        for (int64_t a = 2; a * a <= M; ++a) {
+            if (M % a || M / a > 1600) continue;
+            FftPlan t1, t2;
+            std::vector<float2> scratch_tw;
+            if (!make_fft_plan(a, false, scratch_tw, t1) || t1.generic) continue;
+            if (!make_fft_plan(M / a, false, scratch_tw, t2) || t2.generic) continue;
+            const int cost = t1.nstages + t2.nstages;
+            if (cost <= best_cost) { best_cost = cost; bestA = a; }
+        }
+        g_radix_cap = 16;
+        return bestA;
+    };
     for (int i : order) {
         const int64_t M = L.bands[i].M;
-        // shared memory per item: padded buffer + two-level twiddle table (two buffers for generic radices)
-        const FftPlan &bf = p->ffts[p->bands[i].fft];
-        const int64_t elems = bf.generic ? 2 * M : M + 16 + bf.tw_count;
         int c = 0;
         while (M > limits[c]) ++c;
-        if (elems * p->cls[c].items_per_cta > smem_cap_elems) {
-            // too long for one CTA: two passes, M = A * B with A the divisor nearest sqrt(M) whose cofactor also plans
-            HugeBand hb;
-            hb.band = i;
-            int64_t bestA = 0;
-            for (int64_t a = 2; a * a <= M; ++a)
-                if (M % a == 0) {
-                    FftPlan t1, t2;
-                    std::vector<float2> scratch_tw;
-                    if (a <= 1600 && M / a <= 1600 && make_fft_plan(a, false, scratch_tw, t1) && !t1.generic &&
-                        make_fft_plan(M / a, false, scratch_tw, t2) && !t2.generic)
-                        bestA = a;
-                }
-            if (!bestA) { delete p; return CQT_ERR_UNSUPPORTED; }
-            hb.A = (int)bestA; hb.B = (int)(M / bestA); hb.TW = 16;
-            hb.fft_A = plan_for(hb.A, false); hb.fft_B = plan_for(hb.B, false);
-            hb.tw_m = append_twiddles(tw, M, hb.log_m_c);
-            hb.scratch_off = p->huge_pitch;
-            p->huge_pitch += (M + 7) / 8 * 8;
-            p->huge.push_back(hb);
-            continue;
+        bool single = M <= two_pass_min;
+        int64_t A2 = 0;
+        if (!single) { A2 = split_two_pass(M); single = A2 == 0; }
+        if (single) {
+            g_radix_cap = c <= 1 ? 8 : (c == 2 ? 12 : 16);   // short bands: fewer registers, more CTAs per SM
+            p->bands[i].fft = plan_for(M, false);
+            g_radix_cap = 16;
+            if (p->bands[i].fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
+            // shared memory per item: padded buffer + two-level twiddle table (two buffers for generic radices)
+            const FftPlan &bf = p->ffts[p->bands[i].fft];
+            const int64_t elems = bf.generic ? 2 * M : M + 16 + bf.tw_count;
+            if (elems * p->cls[c].items_per_cta > smem_cap_elems) {
+                A2 = split_two_pass(M);
+                if (!A2) { delete p; return CQT_ERR_UNSUPPORTED; }
+                single = false;
+            } else {
+                p->cls[c].work.push_back(i);
+                p->cls[c].max_elems = (int)std::max<int64_t>(p->cls[c].max_elems, elems);
+                p->cls[c].n_bands++;
+            }
         }
-        p->cls[c].work.push_back(i);
-        p->cls[c].max_elems = (int)std::max<int64_t>(p->cls[c].max_elems, elems);
-        p->cls[c].n_bands++;
+        if (!single) {
+            TwoPassBand tb{};
+            tb.band = i;
+            tb.A = (int32_t)A2;
+            tb.B = (int32_t)(M / A2);
+            g_radix_cap = tp_radix_cap;
+            tb.fft_A = plan_for(tb.A, false, true);
+            tb.fft_B = plan_for(tb.B, false, true);
+            g_radix_cap = 16;
+            int lc = 0;
+            tb.tw_m = append_twiddles(tw, M, lc);
+            tb.log_m_c = lc;
+            tb.n_m = (int32_t)tw.size() - tb.tw_m;
+            tb.scratch_off = p->two_pass_pitch;
+            p->two_pass_pitch += (M + 7) / 8 * 8;
+            TwoPassGroup &g = p->two_pass[(tb.A <= 256 && tb.B <= 256) ? 0 : 1];
+            g.bands.push_back(tb);
+            const int tw_tile = two_pass_tile();
+            g.max_tiles_cols = std::max(g.max_tiles_cols, (tb.B + tw_tile - 1) / tw_tile);
+            g.max_tiles_rows = std::max(g.max_tiles_rows, (tb.A + tw_tile - 1) / tw_tile);
+            g.smem_cols = std::max(g.smem_cols, two_pass_smem_cols(tb));
+            g.smem_rows = std::max(g.smem_rows, two_pass_smem_rows(tb));
+        }
     }
     if (std::getenv("CQT_VERBOSE_PLAN")) {
         std::fprintf(stderr, "cqt plan: N %lld Lp %lld A %lld B %lld fftA %d fftB %d tw_rows %d tw_rows_inv %d tw_cols %d n_lp %d n_n %d "
@@ -304,6 +355,12 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         for (int c = 0; c < kNumClasses; ++c)
             std::fprintf(stderr, "  class %d: bands %d threads %d items %d max_elems %d\n", c, p->cls[c].n_bands, p->cls[c].threads,
                          p->cls[c].items_per_cta, p->cls[c].max_elems);
+        for (int g = 0; g < 2; ++g) {
+            std::fprintf(stderr, "  two-pass group %d: %zu bands, smem %zu / %zu, tiles %d / %d:", g, p->two_pass[g].bands.size(),
+                         p->two_pass[g].smem_cols, p->two_pass[g].smem_rows, p->two_pass[g].max_tiles_cols, p->two_pass[g].max_tiles_rows);
+            for (const auto &b : p->two_pass[g].bands) std::fprintf(stderr, " %dx%d(%d+%d)", b.A, b.B, p->ffts[b.fft_A].nstages, p->ffts[b.fft_B].nstages);
+            std::fprintf(stderr, "\n");
+        }
     }
     if (p->device < 0) { *out = p; return CQT_OK; }
 
@@ -348,7 +405,8 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     chk(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
     if (e == cudaSuccess) chk(configure_band_kernels(*p));
     if (e == cudaSuccess) chk(configure_long_fft_kernels(*p));
-    if (e == cudaSuccess) chk(configure_huge_kernels(*p));
+    for (auto &g : p->two_pass) chk(upload(g.d_recs, g.bands));
+    if (e == cudaSuccess) chk(configure_two_pass_kernels(*p));
     cudaSetDevice(cur);
     if (e != cudaSuccess) { cqt_plan_destroy(p); return CQT_ERR_CUDA; }
     *out = p;
@@ -383,7 +441,7 @@ cqt_status cqt_plan_band_info(const cqt_plan *p, int64_t band, cqt_band_info *ou
 size_t cqt_plan_workspace_bytes(const cqt_plan *p, int64_t batch) {
     if (!p || batch <= 0) return 0;
     const int64_t t = p->lf.A > 1 ? p->lf.Lp : 0;
-    const int64_t per = t + std::max<int64_t>(p->lf.x_pitch, p->y_pitch + p->lf.Lp) + p->huge_pitch;
+    const int64_t per = t + std::max<int64_t>(p->lf.x_pitch, p->y_pitch + p->lf.Lp) + p->two_pass_pitch;
     return (size_t)(256 + batch * per * (int64_t)sizeof(float2));
 }
 
@@ -494,7 +552,7 @@ cqt_status run_analysis_form(const cqt_plan *p, const float *table, const float 
     cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
     if (s != CQT_OK) return s;
     cudaError_t e = launch_rfft_forward(*p, x, x_stride, batch, valid_len, k.T, k.second, k.st);
-    if (e == cudaSuccess) e = launch_huge_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), k.huge, batch, k.st);
+    if (e == cudaSuccess) e = launch_two_pass_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), k.huge, batch, k.st);
     if (e == cudaSuccess) e = launch_bands_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), batch, k.st);
     return end_call(k, e);
 }
@@ -504,7 +562,7 @@ cqt_status run_synthesis_form(const cqt_plan *p, const float *table, bool fold, 
     Call k;
     cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
     if (s != CQT_OK) return s;
-    cudaError_t e = launch_huge_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, k.huge, batch, k.st);
+    cudaError_t e = launch_two_pass_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, k.huge, batch, k.st);
     if (e == cudaSuccess) e = launch_bands_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, batch, k.st);
     if (e == cudaSuccess) e = launch_rfft_inverse(*p, k.second, k.zbuf, k.T, x, x_stride, batch, valid_len, k.st);
     return end_call(k, e);

@@ -162,14 +162,17 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
     return a;
 }
 
-// one instantiation per length class: threads per CTA and CTAs per SM the registers must allow
-#define CQT_CLASS_TABLE(X) X(0, 256, 2, true) X(1, 64, 16, false) X(2, 256, 4, false) X(3, 512, 2, false) X(4, 1024, 1, false)
+// kernel instantiations: (threads per CTA, CTAs per SM the registers must allow, one warp per item)
+#define CQT_KERNEL_TABLE(X) \
+    X(256, 2, true) X(64, 16, false) X(128, 8, false) X(256, 4, false) X(512, 2, false) X(1024, 1, false) \
+    X(128, 4, false) X(256, 2, false) X(512, 1, false) X(256, 3, false) X(768, 2, false) X(1024, 2, false) X(384, 4, false) X(512, 3, false)
 
 template <bool ANALYSIS>
-static const void *class_kernel(int cls) {
-#define X(C, T, B, W) \
-    if (cls == C) return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W> : (const void *)bands_to_spectrum_kernel<T, B, W>;
-    CQT_CLASS_TABLE(X)
+static const void *class_kernel(const BandClass &c) {
+#define X(T, B, W)                                                   \
+    if (c.threads == T && c.min_blocks == B && (c.items_per_cta > 1) == W) \
+        return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W> : (const void *)bands_to_spectrum_kernel<T, B, W>;
+    CQT_KERNEL_TABLE(X)
 #undef X
     return nullptr;
 }
@@ -182,7 +185,9 @@ static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, Ba
     const size_t smem = (size_t)c.max_elems * c.items_per_cta * sizeof(float2);
     const long long grid = (items + c.items_per_cta - 1) / c.items_per_cta;
     void *args[] = {&a};
-    cudaError_t e = cudaLaunchKernel(class_kernel<ANALYSIS>(cls), dim3((unsigned)grid), dim3(c.threads), args, smem, st);
+    const void *fn = class_kernel<ANALYSIS>(c);
+    if (!fn) return cudaErrorInvalidDeviceFunction;
+    cudaError_t e = cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(c.threads), args, smem, st);
     note_launch(p, name, st);
     return e;
 }
@@ -250,9 +255,10 @@ cudaError_t configure_band_kernels(const cqt_plan &p) {
     for (int i = 0; i < kNumClasses; ++i) {
         const size_t s = (size_t)p.cls[i].max_elems * p.cls[i].items_per_cta * sizeof(float2);
         if (s <= 48 * 1024) continue;
-        cudaError_t e = cudaFuncSetAttribute(class_kernel<true>(i), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
+        if (!class_kernel<true>(p.cls[i])) return cudaErrorInvalidDeviceFunction;
+        cudaError_t e = cudaFuncSetAttribute(class_kernel<true>(p.cls[i]), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(class_kernel<false>(i), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
+        e = cudaFuncSetAttribute(class_kernel<false>(p.cls[i]), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

@@ -402,7 +402,7 @@ __device__ __forceinline__ void only_stage(const Tile &t, Load load, Store store
 // caller (stage_twiddles) WITHOUT a barrier after it: the first stage synchronises once its operand loads
 // are issued.  The routine synchronises between stages, not at the end.
 template <int SIGN, class Sync, bool POW2, bool PAD, bool COLFAST_IN, bool REV, bool COLFAST_OUT, bool DIRECT, class Load, class Store>
-__device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, Store store, int tid, int nthr) {
+__device__ __forceinline__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, Store store, int tid, int nthr) {
     const int d = fp.nstages;
     if (d == 1) {
         Sync::sync();   // tables staged by the caller become visible to the functors
@@ -437,7 +437,7 @@ __device__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Lo
 // Same, but every stage after the first runs in shared memory and the results stay there
 // (digit-reversed positions, see dif_pos); ends with a sync.
 template <int SIGN, class Sync, bool POW2, bool COLFAST_IN, bool DIRECT, class Load>
-__device__ void fft_fused_keep(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
+__device__ __forceinline__ void fft_fused_keep(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
     const int d = fp.nstages;
     if (d == 1) {
         auto keep = [&](int k, int col, float2 v) { t.buf[(size_t)k * t.pitch + col] = v; };

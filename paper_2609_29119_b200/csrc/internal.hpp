@@ -16,6 +16,7 @@ constexpr int kNumClasses = 5;
 // Launch shape of one band-length class.
 struct BandClass {
     int threads = 0;         // threads per CTA
+    int min_blocks = 1;      // CTAs per SM the kernel instantiation is compiled for (register budget)
     int items_per_cta = 1;   // > 1: one warp per (band, signal) item
     int max_elems = 0;       // shared-memory elements (float2) per item
     int n_bands = 0;         // bands in the class
@@ -35,13 +36,13 @@ struct LongFft {
     int64_t x_pitch = 0;          // elements per signal of the half-spectrum buffer (Lp + 1 rounded up)
 };
 
-// A band too long for one CTA: M = A * B, two passes through a scratch row of M complex values.
-struct HugeBand {
-    int band = 0;
-    int A = 0, B = 0, TW = 16;
-    int fft_A = -1, fft_B = -1;
-    int tw_m = 0, log_m_c = 0;
-    int64_t scratch_off = 0;   // into one signal's huge-band scratch row
+using TwoPassBand = TwoPassRec;
+
+struct TwoPassGroup {
+    std::vector<TwoPassBand> bands;
+    TwoPassRec *d_recs = nullptr;
+    int max_tiles_cols = 0, max_tiles_rows = 0;
+    size_t smem_cols = 0, smem_rows = 0;
 };
 
 struct DevicePlan {
@@ -70,8 +71,8 @@ struct cqt_plan {
     int y_planes = 1;                  // largest number of bands covering one bin
     cqt::LongFft lf;
     cqt::BandClass cls[cqt::kNumClasses];
-    std::vector<cqt::HugeBand> huge;
-    int64_t huge_pitch = 0;            // scratch elements per signal for the huge bands
+    cqt::TwoPassGroup two_pass[2];     // [0]: both factors <= 256, [1]: larger factors
+    int64_t two_pass_pitch = 0;        // scratch elements per signal for the two-pass bands
     cqt::DevicePlan d;
     int max_smem_optin = 0;
     int sm_count = 0;
@@ -108,11 +109,14 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
                                      float2 *Y, int64_t batch, cudaStream_t st);
 cudaError_t configure_band_kernels(const cqt_plan &p);
 
-// band_huge.cu
-cudaError_t launch_huge_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c, float2 *scratch,
-                                      int64_t batch, cudaStream_t st);
-cudaError_t launch_huge_to_spectrum(const cqt_plan &p, const float *table, bool fold, const float2 *c, float2 *Y,
-                                    float2 *scratch, int64_t batch, cudaStream_t st);
-cudaError_t configure_huge_kernels(const cqt_plan &p);
+// band_two_pass.cu
+cudaError_t launch_two_pass_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
+                                          float2 *scratch, int64_t batch, cudaStream_t st);
+cudaError_t launch_two_pass_to_spectrum(const cqt_plan &p, const float *table, bool fold, const float2 *c, float2 *Y,
+                                        float2 *scratch, int64_t batch, cudaStream_t st);
+cudaError_t configure_two_pass_kernels(const cqt_plan &p);
+size_t two_pass_smem_cols(const TwoPassBand &b);
+size_t two_pass_smem_rows(const TwoPassBand &b);
+int two_pass_tile();
 
 }  // namespace cqt

@@ -46,6 +46,15 @@ struct BandRec {
     float inv_M;
 };
 
+// A band transformed in two passes (M = A * B) through a scratch row.
+struct TwoPassRec {
+    int32_t band;
+    int32_t A, B;
+    int32_t fft_A, fft_B;        // FftPlan indices (plans with full twiddle tables)
+    int32_t tw_m, log_m_c, n_m;  // two-level table of W_M
+    int64_t scratch_off;         // into one signal's two-pass scratch row
+};
+
 // Per-bin cover: bands cover_lo .. cover_lo + cover_n - 1 contain the bin (contiguous because
 // support starts and ends are monotone in the band index).
 struct BinCover {
