@@ -381,7 +381,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         }
     }
     std::vector<int32_t> cover(N / 2 + 1);
-    for (int64_t k = 0; k <= N / 2; ++k) cover[k] = (L.cover_lo[k] << 8) | L.cover_n[k];
+    for (int64_t k = 0; k <= N / 2; ++k) cover[k] = ((L.cover_lo[k] % p->y_planes) << 8) | L.cover_n[k];
     cudaError_t e = cudaSuccess;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
     chk(upload(p->d.bands, p->bands));

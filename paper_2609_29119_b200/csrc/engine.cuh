@@ -286,11 +286,12 @@ __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, co
         if (active) {
             if (DIRECT) apply_twiddle_direct<R, SIGN>(tw, b, re, im);
             else apply_twiddle_powers<R, SIGN>(tw, fp.logC, b, re, im);
-            float2 *p = t.buf + (size_t)b * t.pitch + col;
+            float2 *p = t.buf + (b * (uint32_t)t.pitch + col);
+            const uint32_t qstep = (uint32_t)spad * (uint32_t)t.pitch;
 #pragma unroll
             for (int q = 0; q < R; ++q)
-                if (CQT_CHK(t.dbg, 101, (size_t)b * t.pitch + col + (size_t)q * spad * t.pitch, t.limit))
-                    p[(size_t)q * spad * t.pitch] = make_float2(re[q], im[q]);
+                if (CQT_CHK(t.dbg, 101, b * t.pitch + col + q * qstep, t.limit))
+                    p[q * qstep] = make_float2(re[q], im[q]);
         }
     }
 }
@@ -307,10 +308,10 @@ __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, c
         const uint32_t np = b - blk * s;
         uint32_t pos = blk * n_cur + np;
         if (PAD) pos += fp.pad_delta ? fastdiv(blk, fp.k1magic[j], fp.k1div[j]) : 0u;
-        float2 *p = t.buf + (size_t)pos * t.pitch + col;
-        const int step = s * t.pitch;
+        float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
+        const uint32_t step = (uint32_t)s * (uint32_t)t.pitch;
         float re[R], im[R];
-        if (!CQT_CHK(t.dbg, 102, (size_t)pos * t.pitch + col + (size_t)(R - 1) * step, t.limit)) continue;
+        if (!CQT_CHK(t.dbg, 102, pos * t.pitch + col + (R - 1) * step, t.limit)) continue;
 #pragma unroll
         for (int q = 0; q < R; ++q) {
             const float2 v = p[q * step];
@@ -363,12 +364,12 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
         }
         uint32_t pos = b * R;
         if (PAD) pos += fp.pad_delta ? fastdiv(b, fp.k1magic[d - 1], fp.k1div[d - 1]) : 0u;
-        const float2 *p = t.buf + (size_t)pos * t.pitch + col;
+        const float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
         float re[R], im[R];
-        if (!CQT_CHK(t.dbg, 103, (size_t)pos * t.pitch + col + (size_t)(R - 1) * t.pitch, t.limit)) continue;
+        if (!CQT_CHK(t.dbg, 103, pos * t.pitch + col + (R - 1) * t.pitch, t.limit)) continue;
 #pragma unroll
         for (int q = 0; q < R; ++q) {
-            const float2 v = p[q * t.pitch];
+            const float2 v = p[q * (uint32_t)t.pitch];
             re[q] = v.x; im[q] = v.y;
         }
         if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);

@@ -53,7 +53,7 @@ struct DevicePlan {
     float *tab_synthesis = nullptr;    // h
     float *tab_analysis_adj = nullptr; // N g / (2 M)
     float *tab_synthesis_adj = nullptr;// h w_k / N
-    int32_t *cover = nullptr;          // per bin: (first covering band << 8) | count
+    int32_t *cover = nullptr;          // per bin: (plane of the first covering band << 8) | number of covering bands
     int *dbg = nullptr;                // 8 status words of the debug-bounds build
 };
 

@@ -57,8 +57,8 @@ struct LongArgs {
     int *dbg;
 };
 
-__device__ __forceinline__ float2 load_packed(const float *row, long long j, int valid_len, int aligned) {
-    const long long i = 2 * j;
+__device__ __forceinline__ float2 load_packed(const float *row, int j, int valid_len, int aligned) {
+    const int i = 2 * j;
     if (i + 1 < valid_len) {
         if (aligned) return __ldg(reinterpret_cast<const float2 *>(row + i));
         return make_float2(__ldg(row + i), __ldg(row + i + 1));
@@ -67,8 +67,8 @@ __device__ __forceinline__ float2 load_packed(const float *row, long long j, int
     return make_float2(0.f, 0.f);
 }
 
-__device__ __forceinline__ void store_packed(float *row, long long j, float2 v, int valid_len, int aligned) {
-    const long long i = 2 * j;
+__device__ __forceinline__ void store_packed(float *row, int j, float2 v, int valid_len, int aligned) {
+    const int i = 2 * j;
     if (i + 1 < valid_len) {
         if (aligned) *reinterpret_cast<float2 *>(row + i) = v;
         else { row[i] = v.x; row[i + 1] = v.y; }
@@ -103,11 +103,11 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     float2 *T = a.T + (long long)ch * a.t_pitch;
     const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
     auto load = [&](int j1, int c) -> float2 {
-        return load_packed(row, (long long)j1 * a.B + j2_0 + c, a.valid_len, a.aligned);
+        return load_packed(row, j1 * a.B + j2_0 + c, a.valid_len, a.aligned);
     };
     auto store = [&](int k1, int c, float2 v) {
         const float2 w = twiddle_s(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
-        if (CQT_CHK(a.dbg, 201, (long long)k1 * a.B + j2_0 + c, a.Lp)) T[(long long)k1 * a.B + j2_0 + c] = cmul(v, w);
+        if (CQT_CHK(a.dbg, 201, k1 * a.B + j2_0 + c, a.Lp)) T[k1 * a.B + j2_0 + c] = cmul(v, w);
     };
     fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
 }
@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     } else {
         const float2 *T = a.T + (long long)ch * a.t_pitch;
         auto load = [&](int j2, int r) -> float2 {
-            const long long i = (long long)row_of(t, r, TW, A) * B + j2;
+            const int i = row_of(t, r, TW, A) * B + j2;
             return CQT_CHK(a.dbg, 202, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
         };
         fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
@@ -170,8 +170,8 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
         if (!CQT_CHK(a.dbg, 203, k, a.Lp) || !CQT_CHK(a.dbg, 204, (size_t)posp * pitch + rpp, B * pitch) ||
             !CQT_CHK(a.dbg, 209, (size_t)pos * pitch + r, B * pitch))
             continue;
-        const float2 z = buf[(size_t)pos * pitch + r];
-        const float2 zp = buf[(size_t)posp * pitch + rpp];
+        const float2 z = buf[pos * (uint32_t)pitch + r];
+        const float2 zp = buf[posp * (uint32_t)pitch + rpp];
         // X_k = 1/2 (1 - i w) Z_k + 1/2 (1 + i w) conj Z_{Lp-k},  w = exp(-2 pi i k / N)
         const float2 w = twiddle_s(wn, a.log_n_c, (uint32_t)k);
         const float2 ev = make_float2(0.5f * (z.x + zp.x), 0.5f * (z.y - zp.y));   // (Z + conj Zp)/2
@@ -187,16 +187,18 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
 // sum over the bands covering bin k, in band order
 __device__ __forceinline__ float2 gather_bin(const LongArgs &a, const float2 *__restrict__ Y, int k) {
     if (!CQT_CHK(a.dbg, 205, k, a.Lp + 1)) return make_float2(0.f, 0.f);
-    const int32_t cv = __ldg(a.cover + k);
-    const int lo = cv >> 8, n = cv & 255;
+    const int32_t cv = __ldg(a.cover + k);     // (plane of the first covering band << 8) | number of covering bands
+    const int n = cv & 255;
     if (!CQT_CHK(a.dbg, 206, n, a.planes + 1)) return make_float2(0.f, 0.f);
-    int plane = lo - (int)fastdiv(lo, a.planes_magic, a.planes) * a.planes;
+    const int plane_len = (int)a.y_plane, wrap = a.planes * plane_len;
+    int off = (cv >> 8) * plane_len + k;
     float2 acc = make_float2(0.f, 0.f);
     for (int i = 0; i < n; ++i) {
-        const float2 v = __ldg(Y + (long long)plane * a.y_plane + k);
+        const float2 v = __ldg(Y + off);
         acc.x += v.x;
         acc.y += v.y;
-        if (++plane == a.planes) plane = 0;
+        off += plane_len;
+        if (off >= wrap) off -= wrap;
     }
     return acc;
 }
@@ -248,7 +250,7 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     const float2 *Z = a.Z + (long long)ch * a.t_pitch;
     const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
     auto load = [&](int q2, int r) -> float2 {
-        const long long i = (long long)(direct ? 0 : t * TW + r) + (long long)A * q2;
+        const int i = (direct ? 0 : t * TW + r) + A * q2;
         return CQT_CHK(a.dbg, 210, i, a.Lp) ? __ldg(Z + i) : make_float2(0.f, 0.f);
     };
     fft_fused_keep<+1, BlockSync, true, true, true>(tile, fp, tws, load, tid, nthr);
@@ -260,9 +262,9 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
         for (int e = tid; e < ncols * B; e += nthr) {
             const int r = e >> a.log_b, j2 = e - (r << a.log_b);
             const int q1 = t * TW + r;
-            const float2 v = buf[(size_t)dif_pos_pow2(fp, j2) * pitch + r];
+            const float2 v = buf[dif_pos_pow2(fp, j2) * (uint32_t)pitch + r];
             const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
-            if (CQT_CHK(a.dbg, 207, (long long)q1 * B + j2, a.Lp)) T[(long long)q1 * B + j2] = cmul(v, w);
+            if (CQT_CHK(a.dbg, 207, q1 * B + j2, a.Lp)) T[q1 * B + j2] = cmul(v, w);
         }
     }
 }
@@ -281,11 +283,11 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     float *row = a.x_out + (long long)ch * a.x_stride;
     const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
     auto load = [&](int q1, int c) -> float2 {
-        const long long i = (long long)q1 * a.B + j2_0 + c;
+        const int i = q1 * a.B + j2_0 + c;
         return CQT_CHK(a.dbg, 208, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
     };
     auto store = [&](int j1, int c, float2 v) {
-        store_packed(row, (long long)j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned);
+        store_packed(row, j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned);
     };
     fft_fused<+1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
 }
