@@ -119,7 +119,7 @@ class ClockSampler:
             q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
                  "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
                  "clocks_event_reasons.sw_power_cap")
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "50",
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "20",
                                           "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -170,9 +170,18 @@ def kernel_algorithmic_bytes(plan, w, batch):
            "irfft_cols": sig if two_pass else 0, "irfft_rows": 0 if two_pass else sig}
     for c in cls_m:
         b = 8 * cls_m[c] * batch + 4 * cls_s[c]
-        out[f"bands_from_spectrum/class{c}"] = b
-        out[f"bands_to_spectrum/class{c}"] = b
+        if c < 0:      # bands on the two-pass kernels: pass 2 writes (analysis) / pass 1 reads (synthesis) the coefficients
+            out["band2p_rows/analysis"] = b
+            out["band2p_cols/synthesis"] = b
+        else:
+            out[f"bands_from_spectrum/class{c}"] = b
+            out[f"bands_to_spectrum/class{c}"] = b
     return out
+
+
+def path_algorithmic_bytes(plan, w, batch, second_is_adjoint=False):
+    """Whole step: signal in, coefficients out, coefficients in, signal out, window tables once per transform."""
+    return 2 * 4 * w.valid_len * batch + 2 * 8 * plan.coeff_count * batch + 2 * 4 * plan.table_length
 
 
 def run_ours(args, w):
@@ -199,9 +208,16 @@ def run_ours(args, w):
     ws = plan.workspace(batch)
     stream = torch.cuda.current_stream()
 
+    adjoint_step = (w.name == "config3")     # that workload is forward analysis + its adjoint on a random cotangent
+    if adjoint_step:
+        cbar = torch.from_numpy(wl.make_cotangent(w, plan.coeff_count)).to(dev)
+
     def step():
         plan.analyse(x, valid_len=w.valid_len, out=c, ws=ws, stream=stream)
-        plan.synthesise(c, valid_len=w.valid_len, out=xr, ws=ws, stream=stream)
+        if adjoint_step:
+            plan.analyse_adjoint(cbar, valid_len=w.valid_len, out=xr, ws=ws, stream=stream)
+        else:
+            plan.synthesise(c, valid_len=w.valid_len, out=xr, ws=ws, stream=stream)
 
     def step_e2e():
         x.copy_(x_host, non_blocking=True)
@@ -233,6 +249,8 @@ def run_ours(args, w):
         step()
     torch.cuda.synchronize()
     # correctness guard of the timed configuration: fp32 round trip >= 120 dB on every channel
+    if adjoint_step:
+        plan.synthesise(c, valid_len=w.valid_len, out=xr, ws=ws, stream=stream)
     xd, xrd = x.double(), xr.double()
     snr = 10 * torch.log10((xd * xd).sum(1) / ((xd - xrd) ** 2).sum(1))
     snr_min = float(snr.min().item())
@@ -275,10 +293,10 @@ def run_ours(args, w):
                    "alg_gbs": alg.get(n, 0) / (v[1] / v[0] * 1e-3) / 1e9} for n, v in per.items()}
     dom = max(per, key=lambda n: per[n][1])
     dom_gbs = kernels[dom]["alg_gbs"]
-    path_bytes = sum(alg.values())
+    path_bytes = path_algorithmic_bytes(plan, w, batch)
     path_gbs = path_bytes / (ms / K * 1e-3) / 1e9
     traffic = None
-    prof = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    prof = os.path.join(ROOT, "profiles", "dram_traffic_workload2.txt")
     if os.path.exists(prof):
         try:
             traffic = json.load(open(prof)).get(w.name, {}).get(dom)
@@ -298,7 +316,8 @@ def run_ours(args, w):
         "config": {"workload": w.name, "channels_per_gpu": batch, "valid_len": w.valid_len, "N": w.N,
                    "bins_per_octave": w.bins_per_octave, "bands": plan.num_bands, "coeffs_per_channel": plan.coeff_count,
                    "round_trips_per_s": batch * world / (ms / K / 1e3), "l2": "inputs larger than L2 (no flush)",
-                   "multi_gpu": "replicas only", "round_trip_snr_db_min": snr_min},
+                   "multi_gpu": "replicas only", "round_trip_snr_db_min": snr_min,
+                   "step": "cqt_analyse + cqt_analyse_adjoint" if adjoint_step else "cqt_analyse + cqt_synthesise"},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
@@ -315,10 +334,57 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_stream(args, w):
+    """Sliced streaming workload: the whole stereo stream is pushed through one SliCQ object in pushes of
+    `hops` half-slices and pulled after every push; reports stream samples per second and slices per second."""
+    import torch
+
+    from paper_2609_29119_b200 import Plan, SliCQ
+    torch.cuda.set_device(0)
+    plan = Plan(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, m_policy=w.m_policy, min_win=w.min_win, device=0)
+    x = torch.from_numpy(wl.make_signal(w)).cuda()
+    n, H = x.shape[1], w.slice_len // 2
+    out = torch.empty((w.channels, n + 2 * w.slice_len), device="cuda")
+    res = {}
+    for label, hops in (("bulk_64_hops_per_push", 64), ("one_hop_per_push", 1)):
+        sq = SliCQ(plan, w.channels, w.transition, max(2, hops + 1))
+
+        def run_once():
+            sq.reset()
+            got = pos = 0
+            while pos < n:
+                m = min(hops * H, n - pos)
+                sq.push(x[:, pos:pos + m])
+                pos += m
+                got += sq.pull(out[:, got:])
+            sq.flush()
+            got += sq.pull(out[:, got:])
+            return got
+        run_once()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        got = run_once()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        xd, yd = x.double(), out[:, :n].double()
+        snr = float((10 * torch.log10((xd * xd).sum(1) / ((xd - yd) ** 2).sum(1))).min())
+        slices = (n + H - 1) // H + 1
+        res[label] = {"ms_total": ms, "msamples_per_s": w.channels * n / ms / 1e3, "slices_per_s": slices * w.channels / ms * 1e3,
+                      "device_bytes": sq.device_bytes(), "snr_db_min": snr, "frames_out": got}
+        sq.close()
+    line = {"metric": "slicq_stream_throughput", "value": res["bulk_64_hops_per_push"]["msamples_per_s"], "unit": UNIT,
+            "n_gpus": 1, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "channels": w.channels, "stream_samples": n, "slice_len": w.slice_len,
+                       "transition": w.transition, "bins_per_octave": w.bins_per_octave}, "stream": res}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2", choices=sorted(wl.CONFIGS))
@@ -331,6 +397,8 @@ def main():
         w = wl.scaled(w, channels=args.channels)
     if args.impl == "reference":
         run_reference(args, w)
+    elif w.slice_len:
+        run_stream(args, w)
     else:
         run_ours(args, w)
 

@@ -83,7 +83,7 @@ typedef struct {
     int64_t coeff_offset; /* into one signal's coefficient row */
     int64_t table_offset; /* into the g / h tables returned by cqt_plan_tables */
     int is_sideband;      /* 0 regular, 1 DC, 2 Nyquist */
-    int launch_class;     /* which of the band kernels' length classes (0 = shortest) runs this band */
+    int launch_class;     /* which of the band kernels' length classes (0 = shortest) runs this band; -1: two-pass kernels */
 } cqt_band_info;
 
 typedef struct cqt_plan cqt_plan;

@@ -431,7 +431,7 @@ cqt_status cqt_plan_band_info(const cqt_plan *p, int64_t band, cqt_band_info *ou
     const HostBand &hb = p->lay.bands[band];
     out->centre_hz = hb.centre_hz; out->centre_bin = hb.kc; out->support = hb.S; out->first_offset = hb.d0;
     out->M = hb.M; out->coeff_offset = hb.coeff_off; out->table_offset = hb.tab_off; out->is_sideband = hb.side;
-    out->launch_class = 0;
+    out->launch_class = -1;   // two-pass bands belong to no single-CTA class
     for (int c = 0; c < kNumClasses; ++c)
         for (int32_t b : p->cls[c].work)
             if (b == band) out->launch_class = c;
