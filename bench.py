@@ -156,6 +156,22 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Largest `value` of any rank (the job's step time is the slowest replica's); identity on one rank."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(samples_per_rank: float, world: int, ms_total: float, steps: int) -> float:
+    """Whole-job Msamples/s of `world` independent replicas given the slowest rank's time for `steps` steps."""
+    return samples_per_rank * world / (ms_total / steps / 1e3) / 1e6
+
+
 def kernel_algorithmic_bytes(plan, w, batch):
     """Minimal HBM bytes each kernel is responsible for per launch: signal samples, coefficients and window
     tables; the packed spectrum, the half spectrum and the weighted-bin rows are intermediates (0 bytes)."""
@@ -237,12 +253,7 @@ def run_ours(args, w):
             fn()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dev)
 
     W, K = max(3, args.warmup), args.steps
     for _ in range(W):
@@ -277,9 +288,8 @@ def run_ours(args, w):
         step_e2e()
     ms_e2e = timed(step_e2e, K)
 
-    samples = float(batch) * w.valid_len * world
-    value = samples / (ms / K / 1e3) / 1e6
-    e2e_value = samples / (ms_e2e / K / 1e3) / 1e6
+    value = job_throughput(float(batch) * w.valid_len, world, ms, K)
+    e2e_value = job_throughput(float(batch) * w.valid_len, world, ms_e2e, K)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
