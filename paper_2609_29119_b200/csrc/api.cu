@@ -306,7 +306,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
             if (p->bands[i].fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
             // shared memory per item: padded buffer + two-level twiddle table (two buffers for generic radices)
             const FftPlan &bf = p->ffts[p->bands[i].fft];
-            const int64_t elems = bf.generic ? 2 * M : M + 16 + bf.tw_count;
+            const int64_t elems = bf.generic ? 2 * M + bf.radix[0] : M + 16 + bf.tw_count;
             if (elems * p->cls[c].items_per_cta > smem_cap_elems) {
                 A2 = split_two_pass(M);
                 if (!A2) { delete p; return CQT_ERR_UNSUPPORTED; }

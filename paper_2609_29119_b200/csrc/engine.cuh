@@ -89,29 +89,37 @@ __device__ __forceinline__ void dif_stage(float2 *buf, int pitch, int ncols, uin
 }
 
 // Generic first stage for a radix with no codelet (a large prime factor): every output is a
-// direct sum over the p inputs of its butterfly; written to `alt`, then copied back.
+// direct sum over the p inputs of its butterfly; written to `alt`, then copied back.  `wp` (p entries of
+// shared memory) receives the table exp(-+2 pi i x / p) first, so the inner loop is two shared loads and a MAC.
 template <int SIGN, class Sync>
-__device__ void dif_stage_generic(float2 *buf, float2 *alt, int pitch, int ncols, int M, int p,
+__device__ void dif_stage_generic(float2 *buf, float2 *alt, float2 *wp, int pitch, int ncols, int M, int p,
                                   const float2 *__restrict__ tw, int logC, int tid, int nthr) {
     const int s = M / p;
     const int tstep = M / p;  // W_p^x = W_M^{x * M/p}
+    for (int x = tid; x < p; x += nthr) {
+        float2 t = twiddle(tw, logC, (uint32_t)x * tstep);
+        if (SIGN > 0) t.y = -t.y;
+        wp[x] = t;
+    }
+    Sync::sync();
     for (int w = tid; w < M * ncols; w += nthr) {
         const int e = w / ncols, col = w - e * ncols;
         const int kq = e / s, np = e - kq * s;
-        float2 acc = make_float2(0.f, 0.f);
+        float ax = 0.f, ay = 0.f;
         int x = 0;
+        const float2 *src = buf + (size_t)np * pitch + col;
+        const int step = s * pitch;
         for (int q = 0; q < p; ++q) {
-            float2 t = twiddle(tw, logC, (uint32_t)x * tstep);
-            if (SIGN > 0) t.y = -t.y;
-            const float2 v = buf[(size_t)(q * s + np) * pitch + col];
-            acc.x += v.x * t.x - v.y * t.y;
-            acc.y += v.x * t.y + v.y * t.x;
+            const float2 t = wp[x];
+            const float2 v = src[(size_t)q * step];
+            ax = fmaf(v.x, t.x, ax); ax = fmaf(-v.y, t.y, ax);
+            ay = fmaf(v.x, t.y, ay); ay = fmaf(v.y, t.x, ay);
             x += kq;
             if (x >= p) x -= p;
         }
         float2 t = twiddle(tw, logC, (uint32_t)np * kq);
         if (SIGN > 0) t.y = -t.y;
-        alt[(size_t)e * pitch + col] = cmul(acc, t);
+        alt[(size_t)e * pitch + col] = cmul(make_float2(ax, ay), t);
     }
     Sync::sync();
     for (int w = tid; w < M * ncols; w += nthr) {
@@ -147,7 +155,7 @@ __device__ void fft_dif(float2 *buf, float2 *alt, int pitch, int ncols, uint32_t
                 CQT_STAGE(2) CQT_STAGE(3) CQT_STAGE(4) CQT_STAGE(5) CQT_STAGE(6) CQT_STAGE(8) CQT_STAGE(9)
                 CQT_STAGE(10) CQT_STAGE(12) CQT_STAGE(15) CQT_STAGE(16)
                 default:
-                    dif_stage_generic<SIGN, Sync>(buf, alt, pitch, ncols, M, r, tw, logC, tid, nthr);
+                    dif_stage_generic<SIGN, Sync>(buf, alt, alt + (size_t)M * pitch, pitch, ncols, M, r, tw, logC, tid, nthr);
                     break;
             }
         }
