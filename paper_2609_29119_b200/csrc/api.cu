@@ -251,7 +251,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     // share an SM (64 registers per thread) except for the longest bands, which fill its shared memory
     int limits[kNumClasses] = {128, 1024, 4096, 13500, 1 << 30};
     int threads[kNumClasses] = {256, 64, 256, 512, 1024};
-    int minb[kNumClasses] = {2, 16, 4, 2, 1};
+    int minb[kNumClasses] = {4, 16, 4, 2, 1};
     // tuning hooks (experiments): CQT_CLASSk="limit,threads,min_blocks", CQT_MAX_RADIX=r
     for (int c = 0; c < kNumClasses; ++c) {
         char name[32];

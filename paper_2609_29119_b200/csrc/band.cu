@@ -164,7 +164,7 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
 
 // kernel instantiations: (threads per CTA, CTAs per SM the registers must allow, one warp per item)
 #define CQT_KERNEL_TABLE(X) \
-    X(256, 2, true) X(64, 16, false) X(256, 4, false) X(512, 2, false) X(1024, 1, false) X(128, 8, false) X(256, 2, false)
+    X(256, 4, true) X(64, 16, false) X(256, 4, false) X(512, 2, false) X(1024, 1, false) X(128, 8, false) X(256, 2, false)
 
 template <bool ANALYSIS>
 static const void *class_kernel(const BandClass &c) {
