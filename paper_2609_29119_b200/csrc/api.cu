@@ -1,6 +1,7 @@
 // Plan construction and the C ABI of the transform calls (see include/cqt.h).
 #include <algorithm>
 #include <cmath>
+#include <complex>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -116,6 +117,56 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp, b
         }
     }
     return true;
+}
+
+// host-side helpers for the chirp-z tables
+void host_fft_pow2(std::vector<std::complex<double>> &v) {   // in-place radix-2, forward sign
+    const size_t n = v.size();
+    for (size_t i = 1, j = 0; i < n; ++i) {
+        size_t bit = n >> 1;
+        for (; j & bit; bit >>= 1) j ^= bit;
+        j ^= bit;
+        if (i < j) std::swap(v[i], v[j]);
+    }
+    for (size_t len = 2; len <= n; len <<= 1) {
+        const double ang = -2.0 * kPi / (double)len;
+        for (size_t i = 0; i < n; i += len)
+            for (size_t k = 0; k < len / 2; ++k) {
+                const std::complex<double> w = std::polar(1.0, ang * (double)k);
+                const std::complex<double> u = v[i + k], t = v[i + k + len / 2] * w;
+                v[i + k] = u + t;
+                v[i + k + len / 2] = u - t;
+            }
+    }
+}
+
+int64_t host_dif_pos(const FftPlan &fp, int64_t k) {
+    int64_t pos = 0, rem = k;
+    for (int j = 0; j < fp.nstages; ++j) { pos = pos * fp.radix[j] + rem % fp.radix[j]; rem /= fp.radix[j]; }
+    return pos;
+}
+
+// chirp exp(-i pi n^2 / M) and the filter spectrum DFT_L(conj chirp, wrapped) / L in the DIF output order of `fl`
+void make_chirp_tables(int64_t M, const FftPlan &fl, std::vector<float2> &tw, FftPlan &fp) {
+    const int64_t L = fl.M;
+    fp.blu_L = (int32_t)L;
+    fp.blu_chirp_off = (int32_t)tw.size();
+    std::vector<std::complex<double>> b(L, 0.0);
+    for (int64_t n = 0; n < M; ++n) {
+        const double ang = -kPi * (double)((n * n) % (2 * M)) / (double)M;
+        tw.push_back(make_float2((float)std::cos(ang), (float)std::sin(ang)));
+        const std::complex<double> c = std::polar(1.0, -ang);   // conj chirp
+        b[n] = c;
+        if (n) b[L - n] = c;
+    }
+    host_fft_pow2(b);
+    fp.blu_filter_off = (int32_t)tw.size();
+    std::vector<float2> perm(L);
+    for (int64_t k = 0; k < L; ++k) {
+        const std::complex<double> v = b[k] / (double)L;
+        perm[host_dif_pos(fl, k)] = make_float2((float)v.real(), (float)v.imag());
+    }
+    tw.insert(tw.end(), perm.begin(), perm.end());
 }
 
 template <class T>
@@ -304,9 +355,23 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
             p->bands[i].fft = plan_for(M, false);
             g_radix_cap = 16;
             if (p->bands[i].fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
-            // shared memory per item: padded buffer + two-level twiddle table (two buffers for generic radices)
+            // a length with a large prime factor is evaluated as a chirp-z transform (two power-of-two transforms
+            // of length L >= 2M - 1 in shared memory) instead of direct sums
+            if (p->ffts[p->bands[i].fft].generic == 1 && p->ffts[p->bands[i].fft].radix[0] >= 32 && M <= 8192 &&
+                !std::getenv("CQT_NO_CHIRP_Z")) {
+                int64_t Lz = 64;
+                while (Lz < 2 * M - 1) Lz *= 2;
+                const int fl = plan_for(Lz, true);
+                FftPlan &bfz = p->ffts[p->bands[i].fft];
+                make_chirp_tables(M, p->ffts[fl], tw, bfz);
+                bfz.blu_fft = fl;
+                bfz.generic = 2;
+            }
+            // shared memory per item: padded buffer + two-level twiddle table (two buffers for generic radices,
+            // the length-L buffer and that plan's table for chirp-z)
             const FftPlan &bf = p->ffts[p->bands[i].fft];
-            const int64_t elems = bf.generic ? 2 * M + bf.radix[0] : M + 16 + bf.tw_count;
+            const int64_t elems = bf.generic == 2 ? bf.blu_L + p->ffts[bf.blu_fft].tw_count
+                                                  : (bf.generic ? 2 * M + bf.radix[0] : M + 16 + bf.tw_count);
             if (elems * p->cls[c].items_per_cta > smem_cap_elems) {
                 A2 = split_two_pass(M);
                 if (!A2) { delete p; return CQT_ERR_UNSUPPORTED; }

@@ -45,6 +45,42 @@ struct Group {
 
 extern __shared__ float2 smem_band[];
 
+// Chirp-z (Bluestein) evaluation of an M-point DFT of sign SIGN whose length has a large prime factor:
+//   X[k] = c[k] sum_n (x[n] c[n]) conj(c[k-n]),  c[n] = exp(SIGN i pi n^2 / M),
+// the convolution through two power-of-two transforms of length L >= 2M - 1 in shared memory: forward DIF
+// (natural -> digit-reversed), product with the precomputed filter spectrum (stored in that order, 1/L included),
+// the DIF network backwards (digit-reversed -> natural).  load(n) yields x[n]; store(k, ., X[k]).
+template <int SIGN, class Sync, class Load, class Store>
+__device__ __forceinline__ void chirp_z_transform(float2 *buf, const FftPlan &fp, const FftPlan *ffts, const float2 *tw,
+                                                  Load load, Store store, int *dbg, int tid, int nthr) {
+    const FftPlan &fl = ffts[fp.blu_fft];
+    const int M = fp.M, L = fp.blu_L;
+    float2 *twl = buf + L;
+    stage_twiddles(twl, tw, fl, tid, nthr);
+    const float2 *chirp = tw + fp.blu_chirp_off;   // exp(-i pi n^2 / M)
+    const float2 *filt = tw + fp.blu_filter_off;
+    const Tile tl{buf, 1, 1, 0u, L, dbg};
+    auto loadc = [&](int n, int) -> float2 {
+        if (n >= M) return make_float2(0.f, 0.f);
+        float2 w = __ldg(chirp + n);
+        if (SIGN > 0) w.y = -w.y;
+        return cmul(load(n, 0), w);
+    };
+    fft_fused_keep<-1, Sync, true, false, false>(tl, fl, twl, loadc, tid, nthr);
+    for (int p = tid; p < L; p += nthr) {
+        float2 f = __ldg(filt + p);
+        if (SIGN > 0) f.y = -f.y;
+        buf[p] = cmul(buf[p], f);
+    }
+    Sync::sync();
+    fft_dit_inverse<Sync>(tl, fl, twl, tid, nthr);
+    for (int k = tid; k < M; k += nthr) {
+        float2 w = __ldg(chirp + k);
+        if (SIGN > 0) w.y = -w.y;
+        store(k, 0, cmul(buf[k], w));
+    }
+}
+
 template <int THREADS, int MINB, bool WARP>
 __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
@@ -78,6 +114,11 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
         return make_float2(g * xv.x, g * xv.y);
     };
     float2 *out = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
+    if (fp.generic == 2) {
+        auto store_c = [&](int n, int, float2 v) { out[n] = v; };
+        chirp_z_transform<+1, Sync>(buf, fp, a.ffts, a.tw, load, store_c, a.dbg, tid, nthr);
+        return;
+    }
     if (fp.generic) {
         float2 *alt = buf + M;
         for (int m = tid; m < M; m += nthr) buf[m] = load(m, 0);
@@ -130,6 +171,10 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
         const float h = __ldg(tab + (d - br.d0));
         if (CQT_CHK(a.dbg, 306, (long long)br.y_off + k, a.y_pitch)) Y[k] = make_float2(h * u.x, h * u.y);
     };
+    if (fp.generic == 2) {
+        chirp_z_transform<-1, Sync>(buf, fp, a.ffts, a.tw, load, store, a.dbg, tid, nthr);
+        return;
+    }
     if (fp.generic) {
         float2 *alt = buf + M;
         for (int n = tid; n < M; n += nthr) buf[n] = load(n, 0);

@@ -402,6 +402,55 @@ __device__ __forceinline__ void only_stage(const Tile &t, Load load, Store store
     }
 }
 
+// One stage of the inverse of the DIF network, run backwards (j = d-1 .. 0): conjugate twiddles first, then the
+// inverse butterfly.  Turns digit-reversed spectra back into natural order; the result is L times the inverse DFT
+// of what a forward (SIGN = -1) DIF run produced.
+template <int R>
+__device__ __forceinline__ void dit_stage(const Tile &t, const FftPlan &fp, const float2 *tw, int j, int n_cur, int tmul,
+                                          int tid, int nthr) {
+    const int s = fp.stride[j];
+    const int total = (fp.M / R) * t.ncols;
+    for (int w = tid; w < total; w += nthr) {
+        const uint32_t b = fastdiv(w, t.ncols_magic, t.ncols);
+        const uint32_t col = w - b * t.ncols;
+        const uint32_t blk = fastdiv(b, fp.smagic[j], s);
+        const uint32_t np = b - blk * s;
+        const uint32_t pos = blk * n_cur + np;
+        float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
+        const uint32_t step = (uint32_t)s * (uint32_t)t.pitch;
+        float re[R], im[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) {
+            const float2 v = p[q * step];
+            re[q] = v.x; im[q] = v.y;
+        }
+        if (s > 1) apply_twiddle_powers<R, +1>(tw, fp.logC, np * tmul, re, im);
+        Codelet<R>::run(im, re);
+#pragma unroll
+        for (int q = 0; q < R; ++q) p[q * step] = make_float2(re[q], im[q]);
+    }
+}
+
+// all stages backwards, in shared memory; power-of-two plans only; ends with a sync
+template <class Sync>
+__device__ void fft_dit_inverse(const Tile &t, const FftPlan &fp, const float2 *tw, int tid, int nthr) {
+    const int d = fp.nstages;
+#pragma unroll 1
+    for (int j = d - 1; j >= 0; --j) {
+        const int n_cur = j == 0 ? fp.M : fp.stride[j - 1];
+        int tmul = 1;
+        for (int i = 0; i < j; ++i) tmul *= fp.radix[i];
+        switch (fp.radix[j]) {
+            case 2: dit_stage<2>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+            case 4: dit_stage<4>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+            case 8: dit_stage<8>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+            case 16: dit_stage<16>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+            default: break;
+        }
+        Sync::sync();
+    }
+}
+
 #define CQT_RADIX_CASES_ALL(X) X(2) X(3) X(4) X(5) X(6) X(8) X(9) X(10) X(12) X(15) X(16)
 #define CQT_RADIX_CASES_POW2(X) X(2) X(4) X(8) X(16)
 

@@ -17,7 +17,7 @@ struct FftPlan {
     int32_t nstages;
     int32_t logC;
     int32_t tw_off;                 // into the plan's twiddle array (float2 elements)
-    int32_t generic;                // 1 if stage 0 is a generic (out-of-place) radix
+    int32_t generic;                // 1: stage 0 is a generic (direct-sum) radix; 2: chirp-z (Bluestein) transform, see blu_*
     int32_t tw_count;               // entries of the two-level table (C + ceil(M / C))
     int32_t pad_delta;              // 1 if single-column buffers skip one element per s_0 positions (bank spread)
     int32_t tw_full_off;            // power-of-two plans: offset of the full table exp(-2 pi i y / M), y < M; else -1
@@ -28,6 +28,11 @@ struct FftPlan {
     int32_t k1div[kMaxStages];      // s_0 / n_j: butterfly blocks of stage j per first-stage output digit
     uint32_t k1magic[kMaxStages];
     int32_t lg[kMaxStages];         // log2 r_j for power-of-two plans
+    // chirp-z evaluation of a length with a large prime factor: two power-of-two transforms of length blu_L
+    int32_t blu_L;                  // power of two >= 2 M - 1
+    int32_t blu_fft;                // FftPlan index of the length-blu_L plan
+    int32_t blu_chirp_off;          // exp(-i pi n^2 / M), n < M, in the twiddle array
+    int32_t blu_filter_off;         // DFT of the conjugate chirp / blu_L, in the digit-reversed order of that plan
 };
 
 // One band of the layout as the kernels see it.
