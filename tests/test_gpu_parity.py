@@ -145,3 +145,49 @@ def test_argument_errors_on_device_plan():
         plan.analyse(x, valid_len=w.N + 2)
     assert e.value.status == -1
     plan.close()
+
+
+def test_unaligned_rows_and_odd_strides():
+    """Signal rows that are not 8-byte aligned (odd element offset, odd stride) take the scalar load/store path."""
+    w = CASES[3]
+    plan = library_plan(w)
+    x = wl.make_signal(w)
+    base = torch.zeros(w.channels * (w.valid_len + 8) + 3, device="cuda")
+    stride = w.valid_len + 7                                   # odd
+    view = base[1:1 + w.channels * stride].view(w.channels, stride)   # starts 4 bytes off an 8-byte boundary
+    view[:, :w.valid_len] = _dev(x)
+    c_ref = plan.analyse(_dev(x), valid_len=w.valid_len)
+    c_un = plan.analyse(view, valid_len=w.valid_len)
+    assert torch.equal(torch.view_as_real(c_ref), torch.view_as_real(c_un))
+    out = torch.full_like(view, 5.0)
+    plan.synthesise(c_ref, valid_len=w.valid_len, out=out)
+    ref = plan.synthesise(c_ref, valid_len=w.valid_len)
+    assert torch.equal(out[:, :w.valid_len], ref)
+    assert torch.all(out[:, w.valid_len:] == 5.0)
+    plan.close()
+
+
+def test_plan_create_default_entry_point_and_tiny_inputs():
+    """cqt_plan_create (multiple-of-4 lengths, current device) and the smallest signals: N = 64, valid_len = 1."""
+    import ctypes as C
+    from paper_2609_29119_b200 import binding as B
+    lib = B.load_library()
+    h = C.c_void_p()
+    assert lib.cqt_plan_create(64.0, 4.0, 32.0, 4, 64, 0, C.byref(h)) == 0
+    assert lib.cqt_plan_signal_length(h) == 64 and lib.cqt_plan_device(h) == torch.cuda.current_device()
+    nb, cc = lib.cqt_plan_num_bands(h), lib.cqt_plan_coeff_count(h)
+    lay = orc.build_layout(64.0, 4.0, 32.0, 4, 64)
+    assert (nb, cc) == (len(lay.bands), lay.coeff_count)
+    ws = torch.empty(lib.cqt_plan_workspace_bytes(h, 2), dtype=torch.uint8, device="cuda")
+    for vl in (64, 1, 63):
+        x = torch.randn(2, vl, device="cuda")
+        c = torch.empty((2, cc), dtype=torch.complex64, device="cuda")
+        y = torch.empty_like(x)
+        st = torch.cuda.current_stream().cuda_stream
+        assert lib.cqt_analyse(h, x.data_ptr(), vl, 2, vl, c.data_ptr(), ws.data_ptr(), ws.numel(), st) == 0
+        assert lib.cqt_synthesise(h, c.data_ptr(), 2, vl, y.data_ptr(), vl, ws.data_ptr(), ws.numel(), st) == 0
+        want = orc.analyse(lay, orc.pad_signal(x.cpu().numpy(), 64))
+        errs = band_rel_errors(lay, c.cpu().numpy(), want)
+        assert errs.max() <= TOL
+        assert snr_db(x.cpu().numpy(), y.cpu().numpy()).min() >= 120.0
+    assert lib.cqt_plan_destroy(h) == 0
