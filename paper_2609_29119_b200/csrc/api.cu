@@ -293,8 +293,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
         br.kc = (int32_t)hb.kc; br.d0 = (int32_t)hb.d0; br.S = (int32_t)hb.S; br.M = (int32_t)hb.M;
         br.tab_off = (int32_t)hb.tab_off; br.coeff_off = (int32_t)hb.coeff_off;
         br.y_off = (int32_t)((int64_t)(i % p->y_planes) * p->y_plane);
-        br.j_lo = (int32_t)hb.j_lo; br.n_in = (int32_t)hb.n_in; br.side = hb.side;
-        br.inv_M = (float)(1.0 / (double)hb.M);
+        br.side = hb.side;
         br.fft = -1;
     }
     // ---- launch classes by band length

@@ -75,8 +75,8 @@ int build_layout(const LayoutDesc &d, HostLayout &L, std::string &why) {
             const int64_t k = kc + d0 + j;
             if (k >= 0 && k <= N / 2) { if (first) { lo = j; first = false; } ++n; }
         }
-        hb.j_lo = lo; hb.n_in = n; hb.y_off = L.y_len;
-        L.table_len += S; L.coeff_count += hb.M; L.y_len += n;
+        hb.j_lo = lo; hb.n_in = n;
+        L.table_len += S; L.coeff_count += hb.M;
         L.bands.push_back(hb);
     };
     auto plateau = [&](int64_t edge, double W, std::vector<double> &g) {

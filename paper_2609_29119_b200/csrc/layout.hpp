@@ -27,7 +27,6 @@ struct HostBand {
     int side;         // 0 regular, 1 DC, 2 Nyquist
     int64_t j_lo;     // first support index with 0 <= kc + d <= N/2
     int64_t n_in;     // number of such entries
-    int64_t y_off;    // running sum of n_in
 };
 
 struct HostLayout {
@@ -37,7 +36,6 @@ struct HostLayout {
     std::vector<double> a;      // N/2 + 1
     int64_t coeff_count = 0;
     int64_t table_len = 0;
-    int64_t y_len = 0;          // sum of n_in
     std::vector<int32_t> cover_lo;  // per bin 0..N/2: first covering band
     std::vector<int32_t> cover_n;   // per bin: number of covering bands
 };

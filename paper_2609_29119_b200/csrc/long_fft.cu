@@ -53,7 +53,7 @@ struct LongArgs {
     int planes;
     const int32_t *cover;
     float scale;
-    uint32_t cols_magic, rows_magic, planes_magic;
+    uint32_t cols_magic, rows_magic;
     int *dbg;
 };
 
@@ -320,7 +320,6 @@ static LongArgs base_args(const cqt_plan &p, int64_t valid_len, int64_t x_stride
     a.y_pitch = p.y_pitch;
     a.y_plane = p.y_plane;
     a.planes = p.y_planes;
-    a.planes_magic = magic_of(p.y_planes);
     a.cover = p.d.cover;
     a.cols_magic = magic_of(a.tw_cols);
     a.dbg = p.d.dbg;

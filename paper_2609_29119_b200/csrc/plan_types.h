@@ -44,11 +44,9 @@ struct BandRec {
     int32_t tab_off;    // into the window tables (S entries, offset order)
     int32_t coeff_off;  // into one signal's coefficient row
     int32_t y_off;      // offset of the band's plane in one signal's weighted-bin scratch (entries indexed by bin)
-    int32_t j_lo;       // first support index whose bin lies in 0..N/2
-    int32_t n_in;       // number of support entries whose bin lies in 0..N/2
     int32_t side;       // 0 regular, 1 DC, 2 Nyquist
-    int32_t fft;        // index of the FftPlan for M
-    float inv_M;
+    int32_t fft;        // index of the FftPlan for M (-1 for bands on the two-pass kernels)
+    int32_t pad_[2];
 };
 
 // A band transformed in two passes (M = A * B) through a scratch row.
