@@ -22,6 +22,7 @@
 // over the bands covering bin k reads planes (lo + i) mod P, i < n, at index k: coalesced, no atomics.
 #include "engine.cuh"
 #include "internal.hpp"
+#include "static_fft.cuh"
 
 namespace cqt {
 
@@ -109,7 +110,8 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
         const float2 w = twiddle_s(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
         if (CQT_CHK(a.dbg, 201, k1 * a.B + j2_0 + c, a.Lp)) T[k1 * a.B + j2_0 + c] = cmul(v, w);
     };
-    fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+    if (TW == 16 && plan_is(fp, 8, 8, 8)) tile_fft3<8, 8, 8, 16, 16, -1, true, false>(buf, tws, load, store, tid, nthr);
+    else fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
 }
 
 // rows owned by CTA t of the forward row kernel: first set TWr*t + i, second set A - TWr*t - TWr + i
@@ -145,8 +147,11 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
             const int i = row_of(t, r, TW, A) * B + j2;
             return CQT_CHK(a.dbg, 202, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
         };
-        fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
+        auto nostore = [](int, int, float2) {};
+        if (TW == 8 && plan_is(fp, 8, 8, 8)) tile_fft3<8, 8, 8, 18, 19, -1, false, true>(buf, tws, load, nostore, tid, nthr);
+        else fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
     }
+    const bool fixed888 = plan_is(fp, 8, 8, 8);
     float2 *X = a.X + (long long)ch * a.x_pitch;
     // epilogue: each thread keeps one owned row (column o) and walks k2; for rows other than k1 = 0 the partner
     // Z_{Lp-k} sits in the mirror row at k2' = B-1-k2, whose position is the digit-wise complement B-1-pos(k2)
@@ -161,7 +166,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     }
     const int k1 = direct ? 0 : row_of(t, r, TW, A);
     for (int k2 = kstart; k2 < B; k2 += kstep) {
-        const uint32_t pos = dif_pos_pow2(fp, k2);
+        const uint32_t pos = fixed888 ? (uint32_t)tile_fft3_pos<8, 8, 8>(k2) : dif_pos_pow2(fp, k2);
         uint32_t posp;
         int rpp = rp;
         if (k1 == 0) { rpp = r; posp = k2 == 0 ? 0u : dif_pos_pow2(fp, B - k2); }
@@ -253,7 +258,10 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
         const int i = (direct ? 0 : t * TW + r) + A * q2;
         return CQT_CHK(a.dbg, 210, i, a.Lp) ? __ldg(Z + i) : make_float2(0.f, 0.f);
     };
-    fft_fused_keep<+1, BlockSync, true, true, true>(tile, fp, tws, load, tid, nthr);
+    auto nostore = [](int, int, float2) {};
+    const bool fixed888 = !direct && TW == 16 && plan_is(fp, 8, 8, 8);
+    if (fixed888) tile_fft3<8, 8, 8, 16, 17, +1, true, true>(buf, tws, load, nostore, tid, nthr);
+    else fft_fused_keep<+1, BlockSync, true, true, true>(tile, fp, tws, load, tid, nthr);
     if (direct) {
         float *row = a.x_out + (long long)ch * a.x_stride;
         for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[dif_pos_pow2(fp, j)], a.valid_len, a.aligned);
@@ -262,7 +270,7 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
         for (int e = tid; e < ncols * B; e += nthr) {
             const int r = e >> a.log_b, j2 = e - (r << a.log_b);
             const int q1 = t * TW + r;
-            const float2 v = buf[dif_pos_pow2(fp, j2) * (uint32_t)pitch + r];
+            const float2 v = buf[(fixed888 ? (uint32_t)tile_fft3_pos<8, 8, 8>(j2) : dif_pos_pow2(fp, j2)) * (uint32_t)pitch + r];
             const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
             if (CQT_CHK(a.dbg, 207, q1 * B + j2, a.Lp)) T[q1 * B + j2] = cmul(v, w);
         }
@@ -289,7 +297,8 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     auto store = [&](int j1, int c, float2 v) {
         store_packed(row, j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned);
     };
-    fft_fused<+1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+    if (TW == 16 && plan_is(fp, 8, 8, 8)) tile_fft3<8, 8, 8, 16, 16, +1, true, false>(buf, tws, load, store, tid, nthr);
+    else fft_fused<+1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
 }
 
 // ---------------------------------------------------------------- host side

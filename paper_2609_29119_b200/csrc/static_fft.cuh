@@ -1,0 +1,97 @@
+// Three-stage tile transform with every stride, radix and column count known at compile time (the common
+// shapes of the long FFT passes: 512 = 8 x 8 x 8 points on 16 or 18 interleaved columns).  Same data flow as the
+// run-time planned engine (first stage from a load functor, middle stage in shared memory, last stage to a
+// store functor or back to shared memory); with constant strides the index arithmetic folds into immediates.
+#pragma once
+#include "engine.cuh"
+
+namespace cqt {
+
+template <int R0, int R1, int R2, int NC, int PITCH, int SIGN, bool COLFAST_IN, bool KEEP, class Load, class Store>
+__device__ __forceinline__ void tile_fft3(float2 *buf, const float2 *twf, Load load, Store store, int tid, int nthr) {
+    constexpr int M = R0 * R1 * R2;
+    constexpr int S0 = R1 * R2;
+    // ---- stage 0: operands from the functor, butterflies over positions b + q S0
+    {
+        constexpr int total = S0 * NC;
+        for (int base = 0; base < total; base += nthr) {
+            const int w = base + tid;
+            const bool active = w < total;
+            const int b = COLFAST_IN ? w / NC : w % S0;
+            const int col = COLFAST_IN ? w % NC : w / S0;
+            float re[R0], im[R0];
+            if (active) {
+#pragma unroll
+                for (int q = 0; q < R0; ++q) {
+                    const float2 v = load(b + q * S0, col);
+                    re[q] = v.x; im[q] = v.y;
+                }
+                if (SIGN < 0) Codelet<R0>::run(re, im); else Codelet<R0>::run(im, re);
+            }
+            if (base == 0) __syncthreads();   // staged tables become visible
+            if (active) {
+                apply_twiddle_direct<R0, SIGN>(twf, (uint32_t)b, re, im);
+                float2 *p = buf + b * PITCH + col;
+#pragma unroll
+                for (int q = 0; q < R0; ++q) p[q * S0 * PITCH] = make_float2(re[q], im[q]);
+            }
+        }
+    }
+    __syncthreads();
+    // ---- stage 1: sub-transforms of length S0, stride R2
+    {
+        constexpr int total = (M / R1) * NC;
+        for (int w = tid; w < total; w += nthr) {
+            const int b = w / NC, col = w % NC;
+            const int blk = b / R2, np = b % R2;
+            float2 *p = buf + (blk * S0 + np) * PITCH + col;
+            float re[R1], im[R1];
+#pragma unroll
+            for (int q = 0; q < R1; ++q) {
+                const float2 v = p[q * R2 * PITCH];
+                re[q] = v.x; im[q] = v.y;
+            }
+            if (SIGN < 0) Codelet<R1>::run(re, im); else Codelet<R1>::run(im, re);
+            apply_twiddle_direct<R1, SIGN>(twf, (uint32_t)(np * R0), re, im);
+#pragma unroll
+            for (int q = 0; q < R1; ++q) p[q * R2 * PITCH] = make_float2(re[q], im[q]);
+        }
+    }
+    __syncthreads();
+    // ---- stage 2: stride 1; butterfly b = k0 R1 + k1 holds frequencies k0 + R0 k1 + R0 R1 q
+    {
+        constexpr int total = (M / R2) * NC;
+        for (int w = tid; w < total; w += nthr) {
+            const int b = w / NC, col = w % NC;
+            float2 *p = buf + (b * R2) * PITCH + col;
+            float re[R2], im[R2];
+#pragma unroll
+            for (int q = 0; q < R2; ++q) {
+                const float2 v = p[q * PITCH];
+                re[q] = v.x; im[q] = v.y;
+            }
+            if (SIGN < 0) Codelet<R2>::run(re, im); else Codelet<R2>::run(im, re);
+            if (KEEP) {
+#pragma unroll
+                for (int q = 0; q < R2; ++q) p[q * PITCH] = make_float2(re[q], im[q]);
+            } else {
+                const int klow = b / R1 + R0 * (b % R1);
+#pragma unroll
+                for (int q = 0; q < R2; ++q) store(klow + q * (R0 * R1), col, make_float2(re[q], im[q]));
+            }
+        }
+    }
+    if (KEEP) __syncthreads();
+}
+
+// position of frequency k after tile_fft3 with KEEP: k = k0 + R0 k1 + R0 R1 k2 sits at (k0 R1 + k1) R2 + k2
+template <int R0, int R1, int R2>
+__device__ __forceinline__ int tile_fft3_pos(int k) {
+    return ((k % R0) * R1 + (k / R0) % R1) * R2 + k / (R0 * R1);
+}
+
+__device__ __forceinline__ bool plan_is(const FftPlan &fp, int r0, int r1, int r2) {
+    return fp.nstages == 3 && fp.radix[0] == r0 && fp.radix[1] == r1 && fp.radix[2] == r2;
+}
+
+}  // namespace cqt
