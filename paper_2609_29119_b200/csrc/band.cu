@@ -186,6 +186,22 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     float2 *tws = buf + M + 16;
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
     const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
+    if (br.side == 0) {
+        // regular band: all bins in range, plane row and table share the support index j = d - d0
+        float2 *Ys = Y + (br.kc + br.d0);
+        const int shift_neg = M + br.d0;
+        auto store_regular = [&](int m, int, float2 u) {
+            const bool lo = m <= last_pos;
+            if (!lo && m < first_neg) return;
+            const int j = lo ? m - br.d0 : m - shift_neg;
+            if (!CQT_CHK(a.dbg, 308, j, br.S)) return;
+            const float h = __ldg(tab + j);
+            Ys[j] = make_float2(h * u.x, h * u.y);
+        };
+        auto load_regular = [&](int n, int) -> float2 { return __ldg(in + n); };
+        fft_fused<-1, Sync, false, true, false, true, false, false>(t, fp, tws, load_regular, store_regular, tid, nthr);
+        return;
+    }
     fft_fused<-1, Sync, false, true, false, true, false, false>(t, fp, tws, load, store, tid, nthr);
 }
 
@@ -248,8 +264,10 @@ struct ForkJoin {
         if (!serial) cudaEventRecord(p.ev_fork, st);
     }
     cudaStream_t stream_for(int cls) {
-        if (serial || cls >= 3 || p.cls[cls].n_bands == 0) return st;
-        const int i = cls == 2 ? 0 : 1;
+        if (serial || cls == 3 || p.cls[cls].n_bands == 0) return st;
+        // the longest bands (one CTA per SM, fewer CTAs than SMs) and the middle class share one helper stream,
+        // the two short classes the other; the 4096 < M <= 13,500 class stays on the caller's stream
+        const int i = (cls == 2 || cls == 4) ? 0 : 1;
         if (!used[i]) { cudaStreamWaitEvent(p.aux[i], p.ev_fork, 0); used[i] = true; }
         return p.aux[i];
     }
