@@ -88,7 +88,51 @@ __device__ __forceinline__ void stage_table(float2 *dst, const float2 *__restric
     for (int i = tid; i < n; i += nthr) dst[i] = __ldg(src + i);
 }
 
+// Every pass exists once as a template over a compile-time Shape (radices, columns, pitch) and is instantiated
+// for the common shapes plus the run-time planned fallback; the kernels pick the instantiation that matches.
+using DynShape = Shape<0, 0, 0, 0, 0>;
+using Sh_8_8_8_16_16 = Shape<8, 8, 8, 16, 16>;
+using Sh_16_16_1_16_16 = Shape<16, 16, 1, 16, 16>;
+using Sh_16_8_1_16_16 = Shape<16, 8, 1, 16, 16>;
+using Sh_16_8_8_8_8 = Shape<16, 8, 8, 8, 8>;
+using Sh_16_16_8_8_8 = Shape<16, 16, 8, 8, 8>;
+using Sh_8_8_8_18_19 = Shape<8, 8, 8, 18, 19>;
+using Sh_16_16_1_18_19 = Shape<16, 16, 1, 18, 19>;
+using Sh_16_8_1_18_19 = Shape<16, 8, 1, 18, 19>;
+using Sh_16_8_8_10_11 = Shape<16, 8, 8, 10, 11>;
+using Sh_8_8_8_16_17 = Shape<8, 8, 8, 16, 17>;
+using Sh_16_16_1_16_17 = Shape<16, 16, 1, 16, 17>;
+using Sh_16_8_1_16_17 = Shape<16, 8, 1, 16, 17>;
+using Sh_16_8_8_8_9 = Shape<16, 8, 8, 8, 9>;
+
+#define CQT_DISPATCH_SHAPES(BODY, FP, NC, ...)                                   \
+    do {                                                                         \
+        if (false) {}                                                            \
+        CQT_SHAPE_LIST(BODY, FP, NC, __VA_ARGS__)                                \
+        else BODY<DynShape>(__VA_ARGS__);                                        \
+    } while (0)
+#define CQT_TRY_SHAPE(BODY, FP, NC, SH, ...) else if (SH::matches(FP, NC)) BODY<SH>(__VA_ARGS__);
+
 // ---------------------------------------------------------------- forward, pass C
+template <class SH>
+__device__ __forceinline__ void cols_fwd_body(const LongArgs &a, const FftPlan &fp, float2 *buf, const float2 *tws,
+                                              const float2 *wl, int j2_0, int ch, int tid, int nthr) {
+    const int TW = a.tw_cols;
+    const float *row = a.x_in + (long long)ch * a.x_stride;
+    float2 *T = a.T + (long long)ch * a.t_pitch;
+    auto load = [&](int j1, int c) -> float2 { return load_packed(row, j1 * a.B + j2_0 + c, a.valid_len, a.aligned); };
+    auto store = [&](int k1, int c, float2 v) {
+        const float2 w = twiddle_s(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
+        if (CQT_CHK(a.dbg, 201, k1 * a.B + j2_0 + c, a.Lp)) T[k1 * a.B + j2_0 + c] = cmul(v, w);
+    };
+    if constexpr (SH::is_static) {
+        tile_fft_static<SH, -1, true, false>(buf, tws, load, store, tid, nthr);
+    } else {
+        const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
+        fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+    }
+}
+
 __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
@@ -100,18 +144,13 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     float2 *wl = tws + fp.M;
     stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
-    const float *row = a.x_in + (long long)ch * a.x_stride;
-    float2 *T = a.T + (long long)ch * a.t_pitch;
-    const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
-    auto load = [&](int j1, int c) -> float2 {
-        return load_packed(row, j1 * a.B + j2_0 + c, a.valid_len, a.aligned);
-    };
-    auto store = [&](int k1, int c, float2 v) {
-        const float2 w = twiddle_s(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
-        if (CQT_CHK(a.dbg, 201, k1 * a.B + j2_0 + c, a.Lp)) T[k1 * a.B + j2_0 + c] = cmul(v, w);
-    };
-    if (TW == 16 && plan_is(fp, 8, 8, 8)) tile_fft3<8, 8, 8, 16, 16, -1, true, false>(buf, tws, load, store, tid, nthr);
-    else fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_16, __VA_ARGS__)          \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_16, __VA_ARGS__)        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_16, __VA_ARGS__)         \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_8, __VA_ARGS__)           \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_8_8_8, __VA_ARGS__)
+    CQT_DISPATCH_SHAPES(cols_fwd_body, fp, TW, a, fp, buf, tws, wl, j2_0, ch, tid, nthr);
 }
 
 // rows owned by CTA t of the forward row kernel: first set TWr*t + i, second set A - TWr*t - TWr + i
@@ -123,22 +162,16 @@ __device__ __forceinline__ int row_of(int t, int r, int TW, int A) {
 }
 
 // ---------------------------------------------------------------- forward, pass R (+ untangle)
-__global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
-    const int tid = threadIdx.x, nthr = blockDim.x;
-    const int ch = blockIdx.y, t = blockIdx.x;
+template <class SH>
+__device__ __forceinline__ void rows_fwd_body(const LongArgs &a, const FftPlan &fp, float2 *buf, const float2 *tws,
+                                              const float2 *wn, int t, int ch, int tid, int nthr) {
     const int A = a.A, B = a.B, TW = a.tw_rows;
     const bool direct = (A == 1);
     const int ncols = direct ? 1 : 2 * TW + 2;
-    const int pitch = direct ? 1 : ncols + 1;   // odd: the transposing accesses are conflict-free
-    const FftPlan &fp = a.ffts[a.fft_B];
-    float2 *buf = smem_long;
-    float2 *tws = buf + (size_t)B * pitch;
-    float2 *wn = tws + fp.M;
-    stage_full(tws, a.tw, fp, tid, nthr);
-    stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
-    const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
+    const int pitch = SH::is_static ? SH::PITCH : (direct ? 1 : ncols + 1);   // odd: conflict-free transposing accesses
     if (direct) {
         const float *row = a.x_in + (long long)ch * a.x_stride;
+        const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
         auto load = [&](int j, int) -> float2 { return load_packed(row, j, a.valid_len, a.aligned); };
         fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
     } else {
@@ -147,11 +180,14 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
             const int i = row_of(t, r, TW, A) * B + j2;
             return CQT_CHK(a.dbg, 202, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
         };
-        auto nostore = [](int, int, float2) {};
-        if (TW == 8 && plan_is(fp, 8, 8, 8)) tile_fft3<8, 8, 8, 18, 19, -1, false, true>(buf, tws, load, nostore, tid, nthr);
-        else fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
+        if constexpr (SH::is_static) {
+            auto nostore = [](int, int, float2) {};
+            tile_fft_static<SH, -1, false, true>(buf, tws, load, nostore, tid, nthr);
+        } else {
+            const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
+            fft_fused_keep<-1, BlockSync, true, false, true>(tile, fp, tws, load, tid, nthr);
+        }
     }
-    const bool fixed888 = plan_is(fp, 8, 8, 8);
     float2 *X = a.X + (long long)ch * a.x_pitch;
     // epilogue: each thread keeps one owned row (column o) and walks k2; for rows other than k1 = 0 the partner
     // Z_{Lp-k} sits in the mirror row at k2' = B-1-k2, whose position is the digit-wise complement B-1-pos(k2)
@@ -166,10 +202,10 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     }
     const int k1 = direct ? 0 : row_of(t, r, TW, A);
     for (int k2 = kstart; k2 < B; k2 += kstep) {
-        const uint32_t pos = fixed888 ? (uint32_t)tile_fft3_pos<8, 8, 8>(k2) : dif_pos_pow2(fp, k2);
+        const uint32_t pos = SH::pos(fp, (uint32_t)k2);
         uint32_t posp;
         int rpp = rp;
-        if (k1 == 0) { rpp = r; posp = k2 == 0 ? 0u : dif_pos_pow2(fp, B - k2); }
+        if (k1 == 0) { rpp = r; posp = k2 == 0 ? 0u : SH::pos(fp, (uint32_t)(B - k2)); }
         else posp = (uint32_t)(B - 1) - pos;
         const int k = k1 + A * k2;
         if (!CQT_CHK(a.dbg, 203, k, a.Lp) || !CQT_CHK(a.dbg, 204, (size_t)posp * pitch + rpp, B * pitch) ||
@@ -186,6 +222,27 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
         X[k] = xk;
         if (k == 0) X[a.Lp] = make_float2(z.x - z.y, 0.f);
     }
+}
+
+__global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int ch = blockIdx.y, t = blockIdx.x;
+    const bool direct = (a.A == 1);
+    const int ncols = direct ? 1 : 2 * a.tw_rows + 2;
+    const int pitch = direct ? 1 : ncols + 1;
+    const FftPlan &fp = a.ffts[a.fft_B];
+    float2 *buf = smem_long;
+    float2 *tws = buf + (size_t)a.B * pitch;
+    float2 *wn = tws + fp.M;
+    stage_full(tws, a.tw, fp, tid, nthr);
+    stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
+#undef CQT_SHAPE_LIST
+#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_18_19, __VA_ARGS__)          \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_18_19, __VA_ARGS__)        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_18_19, __VA_ARGS__)         \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_10_11, __VA_ARGS__)
+    CQT_DISPATCH_SHAPES(rows_fwd_body, fp, ncols, a, fp, buf, tws, wn, t, ch, tid, nthr);
 }
 
 // ---------------------------------------------------------------- inverse: overlap-add + retangle
@@ -239,45 +296,81 @@ __global__ void __launch_bounds__(256) gather_retangle_kernel(LongArgs a) {
 }
 
 // ---------------------------------------------------------------- inverse, pass R'
-__global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
-    const int tid = threadIdx.x, nthr = blockDim.x;
-    const int ch = blockIdx.y, t = blockIdx.x;
+template <class SH>
+__device__ __forceinline__ void rows_inv_body(const LongArgs &a, const FftPlan &fp, float2 *buf, const float2 *tws,
+                                              const float2 *wl, int t, int ch, int tid, int nthr) {
     const int A = a.A, B = a.B, TW = a.tw_rows;
     const bool direct = (A == 1);
     const int ncols = direct ? 1 : TW;
-    const int pitch = direct ? 1 : (TW | 1);
-    const FftPlan &fp = a.ffts[a.fft_B];
-    float2 *buf = smem_long;
-    float2 *tws = buf + (size_t)B * pitch;
-    float2 *wl = tws + fp.M;
-    stage_full(tws, a.tw, fp, tid, nthr);
-    if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
+    const int pitch = SH::is_static ? SH::PITCH : (direct ? 1 : (TW | 1));
     const float2 *Z = a.Z + (long long)ch * a.t_pitch;
-    const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
     auto load = [&](int q2, int r) -> float2 {
         const int i = (direct ? 0 : t * TW + r) + A * q2;
         return CQT_CHK(a.dbg, 210, i, a.Lp) ? __ldg(Z + i) : make_float2(0.f, 0.f);
     };
-    auto nostore = [](int, int, float2) {};
-    const bool fixed888 = !direct && TW == 16 && plan_is(fp, 8, 8, 8);
-    if (fixed888) tile_fft3<8, 8, 8, 16, 17, +1, true, true>(buf, tws, load, nostore, tid, nthr);
-    else fft_fused_keep<+1, BlockSync, true, true, true>(tile, fp, tws, load, tid, nthr);
+    if constexpr (SH::is_static) {
+        auto nostore = [](int, int, float2) {};
+        tile_fft_static<SH, +1, true, true>(buf, tws, load, nostore, tid, nthr);
+    } else {
+        const Tile tile{buf, pitch, ncols, a.rows_magic, B * pitch, a.dbg};
+        fft_fused_keep<+1, BlockSync, true, true, true>(tile, fp, tws, load, tid, nthr);
+    }
     if (direct) {
         float *row = a.x_out + (long long)ch * a.x_stride;
-        for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[dif_pos_pow2(fp, j)], a.valid_len, a.aligned);
+        for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[SH::pos(fp, (uint32_t)j)], a.valid_len, a.aligned);
     } else {
         float2 *T = a.T + (long long)ch * a.t_pitch;
         for (int e = tid; e < ncols * B; e += nthr) {
             const int r = e >> a.log_b, j2 = e - (r << a.log_b);
             const int q1 = t * TW + r;
-            const float2 v = buf[(fixed888 ? (uint32_t)tile_fft3_pos<8, 8, 8>(j2) : dif_pos_pow2(fp, j2)) * (uint32_t)pitch + r];
+            const float2 v = buf[SH::pos(fp, (uint32_t)j2) * (uint32_t)pitch + r];
             const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
             if (CQT_CHK(a.dbg, 207, q1 * B + j2, a.Lp)) T[q1 * B + j2] = cmul(v, w);
         }
     }
 }
 
+__global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int ch = blockIdx.y, t = blockIdx.x;
+    const bool direct = (a.A == 1);
+    const int ncols = direct ? 1 : a.tw_rows;
+    const int pitch = direct ? 1 : (a.tw_rows | 1);
+    const FftPlan &fp = a.ffts[a.fft_B];
+    float2 *buf = smem_long;
+    float2 *tws = buf + (size_t)a.B * pitch;
+    float2 *wl = tws + fp.M;
+    stage_full(tws, a.tw, fp, tid, nthr);
+    if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
+#undef CQT_SHAPE_LIST
+#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_17, __VA_ARGS__)          \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_17, __VA_ARGS__)        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_17, __VA_ARGS__)         \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_9, __VA_ARGS__)
+    CQT_DISPATCH_SHAPES(rows_inv_body, fp, ncols, a, fp, buf, tws, wl, t, ch, tid, nthr);
+}
+
 // ---------------------------------------------------------------- inverse, pass C' (+ unpack)
+template <class SH>
+__device__ __forceinline__ void cols_inv_body(const LongArgs &a, const FftPlan &fp, float2 *buf, const float2 *tws,
+                                              int j2_0, int ch, int tid, int nthr) {
+    const int TW = a.tw_cols;
+    const float2 *T = a.T + (long long)ch * a.t_pitch;
+    float *row = a.x_out + (long long)ch * a.x_stride;
+    auto load = [&](int q1, int c) -> float2 {
+        const int i = q1 * a.B + j2_0 + c;
+        return CQT_CHK(a.dbg, 208, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
+    };
+    auto store = [&](int j1, int c, float2 v) { store_packed(row, j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned); };
+    if constexpr (SH::is_static) {
+        tile_fft_static<SH, +1, true, false>(buf, tws, load, store, tid, nthr);
+    } else {
+        const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
+        fft_fused<+1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+    }
+}
+
 __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
@@ -287,19 +380,16 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)a.A * TW;
     stage_full(tws, a.tw, fp, tid, nthr);
-    const float2 *T = a.T + (long long)ch * a.t_pitch;
-    float *row = a.x_out + (long long)ch * a.x_stride;
-    const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
-    auto load = [&](int q1, int c) -> float2 {
-        const int i = q1 * a.B + j2_0 + c;
-        return CQT_CHK(a.dbg, 208, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
-    };
-    auto store = [&](int j1, int c, float2 v) {
-        store_packed(row, j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned);
-    };
-    if (TW == 16 && plan_is(fp, 8, 8, 8)) tile_fft3<8, 8, 8, 16, 16, +1, true, false>(buf, tws, load, store, tid, nthr);
-    else fft_fused<+1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+#undef CQT_SHAPE_LIST
+#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_16, __VA_ARGS__)          \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_16, __VA_ARGS__)        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_16, __VA_ARGS__)         \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_8, __VA_ARGS__)           \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_8_8_8, __VA_ARGS__)
+    CQT_DISPATCH_SHAPES(cols_inv_body, fp, TW, a, fp, buf, tws, j2_0, ch, tid, nthr);
 }
+#undef CQT_SHAPE_LIST
 
 // ---------------------------------------------------------------- host side
 static uint32_t magic_of(uint32_t d) { return d <= 1 ? 0u : (uint32_t)(((1ull << 32) + d - 1) / d); }
