@@ -15,6 +15,8 @@ Contents
   build_layout          band centres, supports, windows g, lengths M, aggregate
                         weight a_k and dual windows h (Sec. 2; the layout rules
                         the paper leaves open are listed in the docstring)
+  build_layout_bands    the same from any list of band centres and widths
+  multires_bands        band list of the multi-resolution layout of Sec. 4
   dft_direct / fft_radix2 / long_dft       F_N of Eq. (dft)
   analyse / analyse_band                    Eq. (analysis) + (band-spectrum),
                                             short inverse DFT evaluated DIRECTLY
@@ -147,44 +149,70 @@ def support_width(f: float, bins_per_octave: int, N: int, fs: float, min_win: fl
     return max(float(min_win), (f / Q) * N / fs)
 
 
-def build_layout(fs: float, fmin: float, fmax: float, bins_per_octave: int, N: int,
-                 window: int = HANN, policy: int = M_MULT4, min_win: float = 4.0) -> Layout:
-    """Constant-Q band layout on N/2+1 bins.
-
-    What the paper fixes (Sec. 2, Sec. 4): geometric centres with constant Q,
-    centres rounded to Fourier bins, real windows whose supports fit in M slots,
-    DC and Nyquist sidebands completing the cover, a_k and h as in Sec. 2.
-    Readings where it is silent (parity unpinned against the paper):
-      * Q = 1/(2^(1/b) - 2^(-1/b)); total support width W = max(min_win, f/Q * N/fs) bins
-        (this width rule reproduces every length of the paper's Table 1);
-      * centres f_j = fmin 2^(j/b) kept while f_j <= fmax and f_j (1 + 1/(2Q)) <= fs/2;
-      * centre bin = floor(f N/fs + 1/2); support = integer offsets with |d| < W/2 (strict);
-        g[d] = w(d / W);
-      * sidebands are plateau windows: 1 in the middle, falling to 0 at the neighbouring
-        band's centre bin with the mirror image of that band's flank.
-    """
-    if N % 2:
-        raise ValueError("N must be even")
+def constant_q_bands(fs: float, fmin: float, fmax: float, bins_per_octave: int, N: int, min_win: float = 4.0):
+    """Centres f_j = fmin 2^(j/b) kept while f_j <= fmax and f_j (1 + 1/(2Q)) <= fs/2, with their
+    support widths in bins (Sec. 2: geometric centres, constant Q)."""
     b = int(bins_per_octave)
     Q = 1.0 / (math.pow(2.0, 1.0 / b) - math.pow(2.0, -1.0 / b))
-    lay = Layout(N=N, fs=float(fs))
-    regular: List[Band] = []
-    widths: List[float] = []
+    centres, widths = [], []
     j = 0
     while True:
         f = fmin * math.pow(2.0, j / b)
         if f > fmax or f * (1.0 + 1.0 / (2.0 * Q)) > fs / 2.0:
             break
-        W = support_width(f, b, N, fs, min_win)
+        centres.append(f)
+        widths.append(support_width(f, b, N, fs, min_win))
+        j += 1
+    return centres, widths
+
+
+def multires_bands(fs: float, fmin: float, N: int, sections: Sequence[Sequence[int]], min_win: float = 4.0):
+    """Multi-resolution band list (Sec. 4, first paragraph): consecutive sections of (octaves, bins per octave);
+    section s starts at fmin 2^(octaves before it) and holds octaves*b centres f_start 2^(j/b), each with the
+    width f/Q_b of its own resolution.  Returns centres, widths and the octave index of every band (bands of one
+    octave share one coefficient length).  A reading: the paper gives the octave counts and resolutions only."""
+    centres, widths, octave = [], [], []
+    f_start, o = float(fmin), 0
+    for n_oct, b in sections:
+        for j in range(int(n_oct) * int(b)):
+            f = f_start * math.pow(2.0, j / int(b))
+            centres.append(f)
+            widths.append(support_width(f, int(b), N, fs, min_win))
+            octave.append(o + j // int(b))
+        f_start *= math.pow(2.0, int(n_oct))
+        o += int(n_oct)
+    return centres, widths, octave
+
+
+def build_layout_bands(fs: float, N: int, centres: Sequence[float], widths: Sequence[float],
+                       window: int = HANN, policy: int = M_MULT4, groups: Optional[Sequence[int]] = None) -> Layout:
+    """Layout from a list of regular bands (centre in Hz, total support width W in bins), low to high.
+
+    Centre bin = floor(f N/fs + 1/2); support = integer offsets with |d| < W/2 (strict); g[d] = w(d / W).
+    M follows `policy` from the support size; bands with the same `groups` value share the largest M of
+    their group (one coefficient length per octave, Sec. 4).  The DC and Nyquist sidebands are plateau
+    windows: 1 in the middle, falling to 0 at the first / last band's centre bin with the mirror image of
+    that band's flank.  Then a_k and h as in Sec. 2."""
+    if N % 2:
+        raise ValueError("N must be even")
+    if len(centres) == 0 or len(centres) != len(widths):
+        raise ValueError("need one width per centre and at least one band")
+    lay = Layout(N=N, fs=float(fs))
+    regular: List[Band] = []
+    for f, W in zip(centres, widths):
         kc = int(math.floor(f * N / fs + 0.5))
         hw = int(math.ceil(W / 2.0)) - 1          # largest integer strictly below W/2
         d = np.arange(-hw, hw + 1, dtype=np.int64)
         g = window_profile(window, d / W)
-        regular.append(Band(kc=kc, d=d, g=g, M=band_length(len(d), policy), centre_hz=f))
-        widths.append(W)
-        j += 1
-    if not regular:
-        raise ValueError("no band fits between fmin and fmax")
+        regular.append(Band(kc=kc, d=d, g=g, M=band_length(len(d), policy), centre_hz=float(f)))
+    if groups is not None:
+        if len(groups) != len(regular):
+            raise ValueError("need one group per band")
+        biggest = {}
+        for bd, gr in zip(regular, groups):
+            biggest[gr] = max(biggest.get(gr, 0), bd.M)
+        for bd, gr in zip(regular, groups):
+            bd.M = biggest[gr]
     k_first, W_first = regular[0].kc, widths[0]
     k_last, W_last = regular[-1].kc, widths[-1]
     if k_first < 2 or N // 2 - k_last < 2:
@@ -205,6 +233,28 @@ def build_layout(fs: float, fmin: float, fmax: float, bins_per_octave: int, N: i
         if bd.kc + bd.d[0] < 1 or bd.kc + bd.d[-1] > N // 2 - 1:
             raise ValueError("a regular band reaches DC or Nyquist")
     return finish_layout(lay)
+
+
+def build_layout(fs: float, fmin: float, fmax: float, bins_per_octave: int, N: int,
+                 window: int = HANN, policy: int = M_MULT4, min_win: float = 4.0) -> Layout:
+    """Constant-Q band layout on N/2+1 bins.
+
+    What the paper fixes (Sec. 2, Sec. 4): geometric centres with constant Q,
+    centres rounded to Fourier bins, real windows whose supports fit in M slots,
+    DC and Nyquist sidebands completing the cover, a_k and h as in Sec. 2.
+    Readings where it is silent (parity unpinned against the paper):
+      * Q = 1/(2^(1/b) - 2^(-1/b)); total support width W = max(min_win, f/Q * N/fs) bins
+        (this width rule reproduces every length of the paper's Table 1);
+      * centres f_j = fmin 2^(j/b) kept while f_j <= fmax and f_j (1 + 1/(2Q)) <= fs/2;
+      * centre bin = floor(f N/fs + 1/2); support = integer offsets with |d| < W/2 (strict);
+        g[d] = w(d / W);
+      * sidebands are plateau windows: 1 in the middle, falling to 0 at the neighbouring
+        band's centre bin with the mirror image of that band's flank.
+    """
+    centres, widths = constant_q_bands(fs, fmin, fmax, bins_per_octave, N, min_win)
+    if not centres:
+        raise ValueError("no band fits between fmin and fmax")
+    return build_layout_bands(fs, N, centres, widths, window, policy)
 
 
 # --------------------------------------------------------------------------

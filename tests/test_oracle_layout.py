@@ -113,3 +113,54 @@ def test_window_profiles():
     t = np.linspace(0, 0.5, 101)
     s = orc.window_profile(orc.HANN, t) ** 2 + orc.window_profile(orc.HANN, 0.5 - t) ** 2
     assert s.min() >= 0.5 - 1e-12
+
+
+SECTIONS = [(3, 8), (4, 16), (2, 32)]      # octaves, bands per octave (Sec. 4, first paragraph)
+
+
+def test_multires_layout_reproduces_table1():
+    """The multi-resolution band list with one power-of-two length per octave gives the printed band counts,
+    per-octave lengths, sideband lengths and coefficient total of Table 1 (Sec. 4)."""
+    rows, total = _table1()
+    N, fs = 65536, 44100.0
+    c, w, octave = orc.multires_bands(fs, fs / 1024.0, N, SECTIONS)
+    lay = orc.build_layout_bands(fs, N, c, w, orc.HANN, orc.M_POW2, octave)
+    n_pos, m_dc, m_ny, n_tot = total
+    assert len(c) == n_pos and len(lay.bands) == n_pos + 2
+    assert lay.bands[0].M == m_dc and lay.bands[-1].M == m_ny and lay.coeff_count == n_tot
+    for o, (_, nb, f_lo, f_hi, M, b) in enumerate(rows):
+        mine = [bd for bd, oo in zip(lay.bands[1:-1], octave) if oo == o]
+        assert len(mine) == nb and all(bd.M == M for bd in mine)
+        # the printed centres are the cited layout's (stretched so that the last centre nears Nyquist); this
+        # reading stays within one band step of them
+        step = 2.0 ** (1.0 / b)
+        assert 1 / step < mine[0].centre_hz / f_lo < step and 1 / step < mine[-1].centre_hz / f_hi < step
+        # resolution of the octave: neighbouring centres a factor 2^(1/b) apart
+        assert np.allclose(np.diff(np.log2([bd.centre_hz for bd in mine])), 1.0 / b)
+    # supports nest where the resolution doubles: the cover of a bin need not be a contiguous band range
+    acc = np.zeros(N // 2 + 1)
+    for bd in lay.bands:
+        k = bd.kc + bd.d
+        ok = (k >= 0) & (k <= N // 2)
+        assert len(bd.d) <= bd.M
+        np.add.at(acc, k[ok], bd.h[ok] * bd.g[ok])
+    assert np.allclose(acc, 1.0, atol=1e-13)
+
+
+def test_band_list_builder_matches_constant_q():
+    """build_layout is build_layout_bands on the constant-Q list; groups only ever raise M to the group's largest."""
+    fs, N = 22050.0, 1 << 13
+    c, w = orc.constant_q_bands(fs, 40.0, fs / 2, 12, N)
+    a = orc.build_layout(fs, 40.0, fs / 2, 12, N, policy=orc.M_SMOOTH)
+    b = orc.build_layout_bands(fs, N, c, w, orc.HANN, orc.M_SMOOTH)
+    assert [(x.kc, x.M, len(x.d)) for x in a.bands] == [(x.kc, x.M, len(x.d)) for x in b.bands]
+    assert all(np.array_equal(x.g, y.g) and np.array_equal(x.h, y.h) for x, y in zip(a.bands, b.bands))
+    # spacing: f_{j+1} / f_j = 2^(1/12); width = f/Q bins with Q = 1/(2^(1/12) - 2^(-1/12)) = f_j / (f_{j+1} - f_{j-1})
+    assert np.allclose(np.array(c[1:]) / np.array(c[:-1]), 2 ** (1 / 12))
+    assert np.allclose(np.array(w[1:-1]), np.maximum(4.0, (np.array(c[2:]) - np.array(c[:-2])) * N / fs))   # min_win = 4
+    assert max(w) > 100
+    groups = [j // 12 for j in range(len(c))]
+    g = orc.build_layout_bands(fs, N, c, w, orc.HANN, orc.M_SMOOTH, groups)
+    for j, (x, y) in enumerate(zip(b.bands[1:-1], g.bands[1:-1])):
+        same = [b.bands[1 + i].M for i in range(len(c)) if groups[i] == groups[j]]
+        assert y.M == max(same) >= x.M
