@@ -74,6 +74,27 @@ typedef struct {
     int device;           /* CUDA device ordinal; -1 builds a host-only plan (queries and tables only) */
 } cqt_plan_desc;
 
+/*
+ * A plan from an explicit list of regular bands, low to high (any painless non-stationary Gabor layout, Sec. 2;
+ * the multi-resolution layout of Sec. 4 is one, see cqt_multires_bands).  Band i has centre centre_hz[i],
+ * rounded to the bin floor(f L/fs + 1/2), and a window of total width width_bins[i] bins (real valued, >= 2)
+ * sampled symmetrically about that bin at the integer offsets |d| < W/2.  M_i follows m_policy from the
+ * support size; bands with the same group[i] >= 0 share the largest M of their group ("one coefficient length
+ * per octave", Sec. 4); group == NULL or group[i] < 0: the band's own length.  The DC and Nyquist sidebands are
+ * added as in cqt_plan_create.  The arrays are host memory, read during the call only.
+ */
+typedef struct {
+    double fs;                /* sample rate, Hz */
+    int64_t L;                /* N, real samples per transform */
+    int window;               /* cqt_window */
+    int m_policy;             /* cqt_m_policy */
+    int device;               /* CUDA device ordinal; -1 builds a host-only plan */
+    int64_t n_bands;          /* regular bands (>= 1) */
+    const double *centre_hz;  /* [n_bands], centre bins must not descend */
+    const double *width_bins; /* [n_bands] */
+    const int32_t *group;     /* [n_bands] or NULL */
+} cqt_band_list_desc;
+
 typedef struct {
     double centre_hz;
     int64_t centre_bin;   /* k_lambda */
@@ -103,6 +124,18 @@ typedef struct cqt_slicq cqt_slicq;
 cqt_status cqt_plan_create(double fs, double fmin, double fmax, int bins_per_octave, int64_t L,
                            cqt_window window, cqt_plan **out);
 cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out);
+/* Errors as above. */
+cqt_status cqt_plan_create_bands(const cqt_band_list_desc *desc, cqt_plan **out);
+/*
+ * Band list of the multi-resolution layout (Sec. 4, first paragraph): n_sections consecutive sections of
+ * octaves[s] octaves at bins_per_octave[s] bands per octave.  Section s starts at fmin * 2^(octaves before it) and
+ * holds centres f_start * 2^(j/b), each with the width (f/Q_b) L/fs bins (at least min_win; <= 0 means 4) of its own
+ * resolution; group[i] is the octave index counted from fmin.  Host arrays of `capacity` entries (any may be
+ * NULL); *n_bands receives the number of bands whether or not they fit.  Pure host arithmetic.
+ */
+cqt_status cqt_multires_bands(double fs, double fmin, int64_t L, const int *octaves, const int *bins_per_octave,
+                              int n_sections, double min_win, int64_t capacity, double *centre_hz, double *width_bins,
+                              int32_t *group, int64_t *n_bands);
 cqt_status cqt_plan_destroy(cqt_plan *plan);
 
 /* Host-side queries; no device access. */

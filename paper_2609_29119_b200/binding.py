@@ -29,6 +29,12 @@ class PlanDesc(C.Structure):
                 ("device", C.c_int)]
 
 
+class BandListDesc(C.Structure):
+    _fields_ = [("fs", C.c_double), ("L", C.c_int64), ("window", C.c_int), ("m_policy", C.c_int), ("device", C.c_int),
+                ("n_bands", C.c_int64), ("centre_hz", C.POINTER(C.c_double)), ("width_bins", C.POINTER(C.c_double)),
+                ("group", C.POINTER(C.c_int32))]
+
+
 class BandInfo(C.Structure):
     _fields_ = [("centre_hz", C.c_double), ("centre_bin", C.c_int64), ("support", C.c_int64),
                 ("first_offset", C.c_int64), ("M", C.c_int64), ("coeff_offset", C.c_int64),
@@ -38,6 +44,10 @@ class BandInfo(C.Structure):
 EXPORTS = {
     "cqt_plan_create": (C.c_int, [C.c_double, C.c_double, C.c_double, C.c_int, C.c_int64, C.c_int, C.POINTER(C.c_void_p)]),
     "cqt_plan_create_ex": (C.c_int, [C.POINTER(PlanDesc), C.POINTER(C.c_void_p)]),
+    "cqt_plan_create_bands": (C.c_int, [C.POINTER(BandListDesc), C.POINTER(C.c_void_p)]),
+    "cqt_multires_bands": (C.c_int, [C.c_double, C.c_double, C.c_int64, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int,
+                                     C.c_double, C.c_int64, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                     C.POINTER(C.c_int32), C.POINTER(C.c_int64)]),
     "cqt_plan_destroy": (C.c_int, [C.c_void_p]),
     "cqt_plan_num_bands": (C.c_int64, [C.c_void_p]),
     "cqt_plan_coeff_count": (C.c_int64, [C.c_void_p]),
@@ -98,6 +108,19 @@ def _check(status: int, what: str) -> None:
         raise CqtError(status, what)
 
 
+def multires_bands(fs: float, fmin: float, L: int, sections, min_win: float = 4.0):
+    """cqt_multires_bands: (centre_hz, width_bins, octave) lists for sections of (octaves, bins per octave)."""
+    lib = load_library()
+    ns = len(sections)
+    octs = (C.c_int * ns)(*[int(s[0]) for s in sections])
+    bpo = (C.c_int * ns)(*[int(s[1]) for s in sections])
+    n = C.c_int64(0)
+    _check(lib.cqt_multires_bands(fs, fmin, L, octs, bpo, ns, min_win, 0, None, None, None, C.byref(n)), "cqt_multires_bands")
+    c, w, g = (C.c_double * n.value)(), (C.c_double * n.value)(), (C.c_int32 * n.value)()
+    _check(lib.cqt_multires_bands(fs, fmin, L, octs, bpo, ns, min_win, n.value, c, w, g, C.byref(n)), "cqt_multires_bands")
+    return list(c), list(w), list(g)
+
+
 def _stream_ptr(stream) -> int:
     import torch
     if stream is None:
@@ -117,6 +140,30 @@ class Plan:
         desc = PlanDesc(fs, fmin, fmax, bins_per_octave, L, window, m_policy, min_win, device)
         h = C.c_void_p()
         _check(self.lib.cqt_plan_create_ex(C.byref(desc), C.byref(h)), "cqt_plan_create_ex")
+        self._adopt(h, device)
+
+    @classmethod
+    def from_bands(cls, fs: float, L: int, centre_hz, width_bins, group=None, window: int = WIN_HANN,
+                   m_policy: int = M_MULT4, device: Optional[int] = None) -> "Plan":
+        """cqt_plan_create_bands: a plan from an explicit list of regular bands."""
+        self = cls.__new__(cls)
+        self.lib = load_library()
+        if device is None:
+            import torch
+            device = torch.cuda.current_device()
+        n = len(centre_hz)
+        if len(width_bins) != n or (group is not None and len(group) != n):
+            raise ValueError("need one width (and one group) per band centre")
+        c = (C.c_double * n)(*[float(v) for v in centre_hz])
+        w = (C.c_double * n)(*[float(v) for v in width_bins])
+        g = (C.c_int32 * n)(*[int(v) for v in group]) if group is not None else None
+        desc = BandListDesc(fs, L, window, m_policy, device, n, c, w, g)
+        h = C.c_void_p()
+        _check(self.lib.cqt_plan_create_bands(C.byref(desc), C.byref(h)), "cqt_plan_create_bands")
+        self._adopt(h, device)
+        return self
+
+    def _adopt(self, h, device) -> None:
         self.handle = h
         self.device = device
         self.N = int(self.lib.cqt_plan_signal_length(h))

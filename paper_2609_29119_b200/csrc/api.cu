@@ -186,7 +186,7 @@ void free_device(cqt_plan *p) {
     cudaFree(p->d.bands); cudaFree(p->d.ffts); cudaFree(p->d.tw);
     cudaFree(p->d.tab_analysis); cudaFree(p->d.tab_synthesis);
     cudaFree(p->d.tab_analysis_adj); cudaFree(p->d.tab_synthesis_adj);
-    cudaFree(p->d.cover); cudaFree(p->d.dbg);
+    cudaFree(p->d.cover); cudaFree(p->d.dbg); cudaFree(p->d.zero_seg);
     for (auto &c : p->cls) cudaFree(c.d_work);
     for (auto &g : p->two_pass) cudaFree(g.d_recs);
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
@@ -229,11 +229,15 @@ cqt_status cqt_plan_create(double fs, double fmin, double fmax, int bins_per_oct
     return cqt_plan_create_ex(&d, out);
 }
 
+static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out);
+
+static bool length_supported(int64_t N) { return is_pow2(N) && N >= 64 && N <= (1ll << 22); }
+
 cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     if (!desc || !out) return CQT_ERR_INVALID_ARG;
     const int64_t N = desc->L;
     if (N < 0) return CQT_ERR_INVALID_ARG;
-    if (!is_pow2(N) || N < 64 || N > (1ll << 22)) return CQT_ERR_UNSUPPORTED;
+    if (!length_supported(N)) return CQT_ERR_UNSUPPORTED;
     cqt_plan *p = new (std::nothrow) cqt_plan();
     if (!p) return CQT_ERR_CUDA;
     LayoutDesc ld{desc->fs, desc->fmin, desc->fmax, desc->bins_per_octave, N, desc->window, desc->m_policy,
@@ -241,8 +245,46 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     std::string why;
     int rc = build_layout(ld, p->lay, why);
     if (rc != 0) { delete p; return (cqt_status)rc; }
+    return finish_plan(p, N, desc->device, out);
+}
+
+cqt_status cqt_plan_create_bands(const cqt_band_list_desc *desc, cqt_plan **out) {
+    if (!desc || !out || !desc->centre_hz || !desc->width_bins || desc->n_bands < 1 || desc->L < 0) return CQT_ERR_INVALID_ARG;
+    const int64_t N = desc->L;
+    if (!length_supported(N)) return CQT_ERR_UNSUPPORTED;
+    if (desc->n_bands > 100000) return CQT_ERR_UNSUPPORTED;
+    std::vector<BandSpec> specs((size_t)desc->n_bands);
+    for (int64_t i = 0; i < desc->n_bands; ++i)
+        specs[i] = BandSpec{desc->centre_hz[i], desc->width_bins[i], desc->group ? desc->group[i] : -1};
+    cqt_plan *p = new (std::nothrow) cqt_plan();
+    if (!p) return CQT_ERR_CUDA;
+    LayoutDesc ld{desc->fs, 0.0, 0.0, 0, N, desc->window, desc->m_policy, 4.0};
+    std::string why;
+    int rc = build_layout_bands(ld, specs, p->lay, why);
+    if (rc != 0) { delete p; return (cqt_status)rc; }
+    return finish_plan(p, N, desc->device, out);
+}
+
+cqt_status cqt_multires_bands(double fs, double fmin, int64_t L, const int *octaves, const int *bins_per_octave,
+                              int n_sections, double min_win, int64_t capacity, double *centre_hz, double *width_bins,
+                              int32_t *group, int64_t *n_bands) {
+    if (!n_bands || capacity < 0) return CQT_ERR_INVALID_ARG;
+    std::vector<BandSpec> specs;
+    std::string why;
+    int rc = multires_bands(fs, fmin, L, octaves, bins_per_octave, n_sections, min_win > 0 ? min_win : 4.0, specs, why);
+    if (rc != 0) return (cqt_status)rc;
+    *n_bands = (int64_t)specs.size();
+    for (int64_t i = 0; i < std::min<int64_t>(capacity, (int64_t)specs.size()); ++i) {
+        if (centre_hz) centre_hz[i] = specs[i].f;
+        if (width_bins) width_bins[i] = specs[i].W;
+        if (group) group[i] = specs[i].group;
+    }
+    return CQT_OK;
+}
+
+static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out) {
     p->N = N;
-    p->device = desc->device;
+    p->device = device;
     const HostLayout &L = p->lay;
     p->g32.resize(L.table_len);
     p->h32.resize(L.table_len);
@@ -456,6 +498,16 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     chk(upload(p->d.tab_analysis_adj, tTA));
     chk(upload(p->d.tab_synthesis_adj, tSA));
     chk(upload(p->d.cover, cover));
+    // nested supports: the bins of a band's widened range outside its support hold zeros in the band's plane
+    std::vector<int2> zero_seg;
+    for (size_t i = 0; i < L.bands.size(); ++i) {
+        const HostBand &hb = L.bands[i];
+        const int64_t s = hb.kc + hb.d0, en = s + hb.S - 1;
+        if (hb.zl > 0) zero_seg.push_back(make_int2((int)(p->bands[i].y_off + s - hb.zl), (int)hb.zl));
+        if (hb.zr > 0) zero_seg.push_back(make_int2((int)(p->bands[i].y_off + en + 1), (int)hb.zr));
+    }
+    p->n_zero_seg = (int)zero_seg.size();
+    if (p->n_zero_seg) chk(upload(p->d.zero_seg, zero_seg));
     chk(upload(p->d.dbg, std::vector<int>(8, 0)));
     for (auto &c : p->cls) chk(upload(c.d_work, c.work));
     cudaDeviceProp prop;

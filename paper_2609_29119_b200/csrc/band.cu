@@ -295,8 +295,21 @@ cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, co
     return cudaSuccess;
 }
 
+// Zero-fill of the bins between a band's support and its widened range (layouts with nested supports).
+__global__ void __launch_bounds__(128) zero_fill_kernel(float2 *Y, long long y_pitch, const int2 *seg) {
+    const int2 sg = seg[blockIdx.x];
+    float2 *y = Y + (long long)blockIdx.y * y_pitch + sg.x;
+    for (int i = threadIdx.x; i < sg.y; i += blockDim.x) y[i] = make_float2(0.f, 0.f);
+}
+
 cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool fold_sidebands, const float2 *c,
                                      float2 *Y, int64_t batch, cudaStream_t st) {
+    if (p.n_zero_seg > 0) {
+        zero_fill_kernel<<<dim3((unsigned)p.n_zero_seg, (unsigned)batch), 128, 0, st>>>(Y, p.y_pitch, p.d.zero_seg);
+        note_launch(p, "zero_fill", st);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     ForkJoin fj(p, st);
     static const char *names[kNumClasses] = {"bands_to_spectrum/class0", "bands_to_spectrum/class1",
                                               "bands_to_spectrum/class2", "bands_to_spectrum/class3",

@@ -55,6 +55,7 @@ struct DevicePlan {
     float *tab_synthesis_adj = nullptr;// h w_k / N
     int32_t *cover = nullptr;          // per bin: (plane of the first covering band << 8) | number of covering bands
     int *dbg = nullptr;                // 8 status words of the debug-bounds build
+    int2 *zero_seg = nullptr;          // (offset into one signal's weighted-bin scratch, length): bins synthesis zero-fills
 };
 
 }  // namespace cqt
@@ -69,6 +70,7 @@ struct cqt_plan {
     int64_t y_pitch = 0;               // weighted-bin scratch elements per signal (y_planes * y_plane)
     int64_t y_plane = 0;               // elements per plane (N/2 + 1 rounded up)
     int y_planes = 1;                  // largest number of bands covering one bin
+    int n_zero_seg = 0;                // zero-fill segments (layouts with nested supports only)
     cqt::LongFft lf;
     cqt::BandClass cls[cqt::kNumClasses];
     cqt::TwoPassGroup two_pass[2];     // [0]: both factors <= 256, [1]: larger factors

@@ -16,6 +16,13 @@ struct LayoutDesc {
     double min_win;
 };
 
+// One regular band of an explicit band list.
+struct BandSpec {
+    double f;       // centre, Hz
+    double W;       // total support width in bins (real valued)
+    int32_t group;  // bands with the same group >= 0 share the largest M of the group; -1: own length
+};
+
 struct HostBand {
     double centre_hz;
     int64_t kc;       // centre bin
@@ -27,6 +34,7 @@ struct HostBand {
     int side;         // 0 regular, 1 DC, 2 Nyquist
     int64_t j_lo;     // first support index with 0 <= kc + d <= N/2
     int64_t n_in;     // number of such entries
+    int64_t zl, zr;   // bins below / above the support that synthesis zero-fills in this band's plane (nested supports)
 };
 
 struct HostLayout {
@@ -42,6 +50,12 @@ struct HostLayout {
 
 // Returns 0 on success, else a cqt_status error code (-1 invalid, -2 unsupported, -3 bad layout).
 int build_layout(const LayoutDesc &d, HostLayout &out, std::string &why);
+// The same from an explicit list of regular bands, low to high (fmin, fmax, bins_per_octave, min_win of d unused).
+int build_layout_bands(const LayoutDesc &d, const std::vector<BandSpec> &bands, HostLayout &out, std::string &why);
+// Band lists: constant-Q (fmin 2^(j/b)), and consecutive sections of (octaves, bins per octave) (Sec. 4).
+int constant_q_bands(const LayoutDesc &d, std::vector<BandSpec> &out, std::string &why);
+int multires_bands(double fs, double fmin, int64_t N, const int *octaves, const int *bins_per_octave, int n_sections,
+                   double min_win, std::vector<BandSpec> &out, std::string &why);
 
 int64_t band_length(int64_t S, int policy);
 

@@ -6,12 +6,23 @@ from oracle import nsgt_oracle as orc
 
 
 def oracle_layout(w: wl.Workload):
+    if w.sections:
+        c, wd, octave = orc.multires_bands(w.fs, w.fmin, w.N, w.sections, w.min_win)
+        return orc.build_layout_bands(w.fs, w.N, c, wd, w.window, w.m_policy, octave)
+    if w.bands:
+        return orc.build_layout_bands(w.fs, w.N, [b[0] for b in w.bands], [b[1] for b in w.bands], w.window, w.m_policy)
     return orc.build_layout(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, policy=w.m_policy,
                             min_win=w.min_win)
 
 
 def library_plan(w: wl.Workload, device=None):
-    from paper_2609_29119_b200 import Plan
+    from paper_2609_29119_b200 import Plan, multires_bands
+    if w.sections:
+        c, wd, octave = multires_bands(w.fs, w.fmin, w.N, w.sections, w.min_win)
+        return Plan.from_bands(w.fs, w.N, c, wd, octave, window=w.window, m_policy=w.m_policy, device=device)
+    if w.bands:
+        return Plan.from_bands(w.fs, w.N, [b[0] for b in w.bands], [b[1] for b in w.bands], None, window=w.window,
+                               m_policy=w.m_policy, device=device)
     return Plan(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, m_policy=w.m_policy,
                 min_win=w.min_win, device=device)
 

@@ -9,6 +9,8 @@ import pytest
 
 import workloads as wl
 from helpers import oracle_layout, library_plan, small_workload
+import paper_2609_29119_b200 as cq
+from oracle import nsgt_oracle as orc
 from paper_2609_29119_b200 import binding as B
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -81,3 +83,69 @@ def test_error_codes_without_a_device():
     assert lib.cqt_status_string(-3).decode().startswith("band layout")
     out = C.c_void_p()
     assert lib.slicq_create(None, 2, 8, 4, C.byref(out)) == -1
+
+
+TABLE1_SECTIONS = [(3, 8), (4, 16), (2, 32)]
+
+
+def _compare_plan(plan, lay):
+    assert plan.num_bands == len(lay.bands) and plan.coeff_count == lay.coeff_count
+    g, h = plan.tables()
+    offs = lay.coeff_offsets
+    t = 0
+    for i, bd in enumerate(lay.bands):
+        bi = plan.band_info(i)
+        assert (bi.centre_bin, bi.support, bi.first_offset, bi.M, bi.coeff_offset, bi.is_sideband, bi.table_offset) == \
+               (bd.kc, len(bd.d), int(bd.d[0]), bd.M, offs[i], bd.sideband, t)
+        assert np.allclose(g[t:t + len(bd.d)], bd.g, rtol=1e-6, atol=1e-9)
+        assert np.allclose(h[t:t + len(bd.d)], bd.h, rtol=1e-6, atol=1e-12)
+        t += len(bd.d)
+
+
+def test_multires_plan_matches_oracle_and_table1():
+    """cqt_multires_bands + cqt_plan_create_bands against the oracle's own list and layout; the totals are the
+    paper's Table 1 (154 bands, 132,992 coefficients)."""
+    fs, N = 44100.0, 65536
+    c, w, octave = orc.multires_bands(fs, fs / 1024.0, N, TABLE1_SECTIONS)
+    lc, lw, lo = cq.multires_bands(fs, fs / 1024.0, N, TABLE1_SECTIONS)
+    assert np.allclose(lc, c, rtol=1e-14) and np.allclose(lw, w, rtol=1e-14) and list(lo) == list(octave)
+    lay = orc.build_layout_bands(fs, N, c, w, orc.HANN, orc.M_POW2, octave)
+    plan = cq.Plan.from_bands(fs, N, lc, lw, lo, m_policy=cq.M_POW2, device=-1)
+    assert plan.num_bands == 154 and plan.coeff_count == 132992
+    _compare_plan(plan, lay)
+    plan.close()
+    # falling resolution: the wide bands of the second section start below the last narrow bands of the first
+    fs, N = 8192.0, 8192
+    c, w, octave = orc.multires_bands(fs, 100.0, N, [(2, 16), (2, 4)])
+    lay = orc.build_layout_bands(fs, N, c, w, orc.HANN, orc.M_POW2, octave)
+    plan = cq.Plan.from_bands(fs, N, c, w, octave, m_policy=cq.M_POW2, device=-1)
+    _compare_plan(plan, lay)
+    starts = [b.kc + b.d[0] for b in lay.bands[1:-1]]
+    assert min(np.diff(starts)) < 0          # supports do nest
+    plan.close()
+
+
+def test_irregular_band_list_plan_matches_oracle():
+    fs, N = 2048.0, 2048
+    c = list(np.arange(24.0, 200.0, 16.0)) + list(200.0 * 2 ** (np.arange(0, 17) / 8.0))
+    c = [f for f in c if f < 820.0]
+    w = [2.0 * (c[min(i + 1, len(c) - 1)] - c[max(i - 1, 0)]) * N / fs / (2 if 0 < i < len(c) - 1 else 1) for i in range(len(c))]
+    lay = orc.build_layout_bands(fs, N, c, w, orc.BLACKMAN_HARRIS, orc.M_SMOOTH)
+    plan = cq.Plan.from_bands(fs, N, c, w, None, window=cq.WIN_BLACKMAN_HARRIS, m_policy=cq.M_SMOOTH, device=-1)
+    _compare_plan(plan, lay)
+    plan.close()
+
+
+def test_band_list_errors():
+    ok = dict(fs=1024.0, L=1024, centre_hz=[40.0, 80.0, 160.0], width_bins=[60.0, 120.0, 240.0], device=-1)
+    cq.Plan.from_bands(**ok).close()
+    for bad, status in [(dict(centre_hz=[80.0, 40.0, 160.0]), -1),       # descending centres
+                        (dict(width_bins=[60.0, 1.0, 240.0]), -1),        # width below 2 bins
+                        (dict(L=1000), -2),                               # N not a power of two
+                        (dict(centre_hz=[40.0, 80.0, 500.0]), -3),        # last band reaches Nyquist
+                        (dict(centre_hz=[1.0, 80.0, 160.0], width_bins=[2.0, 120.0, 240.0]), -3)]:   # first centre below bin 2
+        with pytest.raises(cq.CqtError) as e:
+            cq.Plan.from_bands(**dict(ok, **bad))
+        assert e.value.status == status
+    # a narrow band nested deep inside a wide neighbour is a legal frame
+    cq.Plan.from_bands(1024.0, 1024, [100.0, 101.0, 200.0], [180.0, 8.0, 200.0], device=-1).close()

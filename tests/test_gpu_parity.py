@@ -34,6 +34,16 @@ CASES = [
     small_workload("n65536_ragged_pow2", N=1 << 16, valid_len=50001, fs=44100.0, fmin=32.70, fmax=22050.0,
                    bins_per_octave=12, m_policy=wl.M_POW2, channels=3),
     wl.scaled(wl.CONFIGS["config3"], channels=2),
+    # band-list plans: the paper's Table 1 layout; falling resolution (nested supports, zero-filled plane bins);
+    # an irregular list (linear then geometric centres)
+    wl.scaled(wl.CONFIGS["table1"], channels=3),
+    small_workload("multires_falling", N=8192, valid_len=8000, fs=8192.0, fmin=100.0, fmax=4096.0, bins_per_octave=0,
+                   m_policy=wl.M_POW2, channels=2, sections=((2, 16), (2, 4))),
+    small_workload("irregular_bands", N=2048, valid_len=2048, fs=2048.0, fmin=24.0, fmax=1024.0, bins_per_octave=0,
+                   window=wl.WIN_BLACKMAN_HARRIS, m_policy=wl.M_SMOOTH, channels=2,
+                   bands=tuple((f, wd) for f, wd in zip(
+                       [24.0 + 16.0 * i for i in range(11)] + [200.0 * 2 ** (i / 8.0) for i in range(17)],
+                       [32.0] * 11 + [200.0 * 2 ** (i / 8.0) * 0.36 for i in range(17)]))),
 ]
 
 

@@ -42,6 +42,10 @@ class Workload:
     slice_len: int = 0
     transition: int = 0
     stream_len: int = 0
+    # band-list layouts: consecutive sections of (octaves, bands per octave) starting at fmin with one coefficient
+    # length per octave (the multi-resolution layout), or explicit (centre Hz, width in bins) pairs
+    sections: tuple = ()
+    bands: tuple = ()
 
 
 CONFIGS = {
@@ -61,6 +65,10 @@ CONFIGS = {
     "config5": Workload("config5", 44100.0, 32.70, 22050.0, 48, 1 << 15, 1 << 15, 2,
                         WIN_HANN, M_SMOOTH, 1005, "pink_notes",
                         slice_len=1 << 15, transition=1 << 13, stream_len=300 * 44100),
+    # the paper's principal configuration (its Table 1): one slice of 2^16 samples, 3/4/2 octaves at 8/16/32 bands per
+    # octave, one power-of-two length per octave; the batch is swept by the benchmark
+    "table1": Workload("table1", 44100.0, 44100.0 / 1024.0, 22050.0, 0, 1 << 16, 1 << 16, 1,
+                       WIN_HANN, M_POW2, 1006, "noise_sines", sections=((3, 8), (4, 16), (2, 32))),
 }
 
 
