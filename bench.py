@@ -458,6 +458,8 @@ def run_stream(args, w):
 
 # the paper's Fig. 2(a): A100 round trip under graph replay, ms per batch size (its Table 2 row is the B = 1 entry)
 PAPER_A100_MS = {1: 0.116, 2: 0.109, 4: 0.131, 8: 0.185, 16: 0.273, 32: 0.461, 64: 0.844, 128: 1.656}
+# its Fig. 2(b): analysis, synthesis, squared loss and backpropagation in eager mode, A100, ms
+PAPER_A100_BACKWARD_MS = {1: 1.969, 2: 1.975, 4: 2.003, 8: 2.012, 16: 2.031, 32: 2.474, 64: 4.601, 128: 8.779}
 
 
 def run_sweep(args, w):
@@ -502,13 +504,23 @@ def run_sweep(args, w):
                     ts.append(e0.elapsed_time(e1))
             return statistics.median(ts)
         eager = median_ms(step, False)
+        # differentiable step (Sec. 5, second experiment): analysis, synthesis, squared loss, backward, eager
+        from paper_2609_29119_b200 import autograd as ad
+        xg = x.clone().requires_grad_(True)
+
+        def train_step():
+            xg.grad = None
+            y = ad.synthesise(plan, ad.analyse(plan, xg))
+            ((y - x) ** 2).sum().backward()
+        backward = median_ms(train_step, False)
         graph = capture_graph(step)
         hot = median_ms(graph.replay, False)
         cold = median_ms(graph.replay, True)
         xd, xrd = x.double(), xr.double()
         snr = float((10 * torch.log10((xd * xd).sum(1) / ((xd - xrd) ** 2).sum(1))).min())
         sweep[str(B)] = {"eager_ms": eager, "graph_ms": hot, "graph_l2_flushed_ms": cold, "snr_db_min": snr,
-                         "paper_a100_graph_ms": PAPER_A100_MS.get(B), "workspace_mb_per_signal": plan.workspace_bytes(B) / B / 1e6,
+                         "paper_a100_graph_ms": PAPER_A100_MS.get(B),
+                         "step_with_backward_eager_ms": backward, "paper_a100_backward_ms": PAPER_A100_BACKWARD_MS.get(B), "workspace_mb_per_signal": plan.workspace_bytes(B) / B / 1e6,
                          "msamples_per_s_l2_flushed": B * w.valid_len / cold / 1e3}
         del graph
     launches = plan.launch_count() - launches0
