@@ -131,6 +131,22 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
     const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
     auto store = [&](int n, int, float2 v) { if (CQT_CHK(a.dbg, 303, n, M)) out[n] = v; };
+    if (br.side == 0) {
+        // regular band: every support bin lies in 1..N/2-1; spectrum and table share the support index j = d - d0
+        const float2 *Xs = X + (br.kc + br.d0);
+        const int shift_neg = M + br.d0;
+        auto load_regular = [&](int m, int) -> float2 {
+            const bool lo = m <= last_pos;
+            if (!lo && m < first_neg) return make_float2(0.f, 0.f);
+            const int j = lo ? m - br.d0 : m - shift_neg;
+            if (!CQT_CHK(a.dbg, 309, j, br.S)) return make_float2(0.f, 0.f);
+            const float g = __ldg(tab + j);
+            const float2 xv = __ldg(Xs + j);
+            return make_float2(g * xv.x, g * xv.y);
+        };
+        fft_fused<+1, Sync, false, true, false, true, false, false>(t, fp, tws, load_regular, store, tid, nthr);
+        return;
+    }
     fft_fused<+1, Sync, false, true, false, true, false, false>(t, fp, tws, load, store, tid, nthr);
 }
 
