@@ -45,6 +45,15 @@ struct Group {
 
 extern __shared__ float2 smem_band[];
 
+// One-CTA-per-item kernels keep the item's radix plan in shared memory: its fields are read inside the stage
+// loops, and a shared-memory copy costs a short-latency load where the global original costs a cache lookup.
+__device__ __forceinline__ const FftPlan &cta_plan(const FftPlan &g, FftPlan &s, int tid, int nthr) {
+    constexpr int kWords = (int)(sizeof(FftPlan) / sizeof(int));
+    for (int i = tid; i < kWords; i += nthr) reinterpret_cast<int *>(&s)[i] = __ldg(reinterpret_cast<const int *>(&g) + i);
+    __syncthreads();
+    return s;
+}
+
 // Chirp-z (Bluestein) evaluation of an M-point DFT of sign SIGN whose length has a large prime factor:
 //   X[k] = c[k] sum_n (x[n] c[n]) conj(c[k-n]),  c[n] = exp(SIGN i pi n^2 / M),
 // the convolution through two power-of-two transforms of length L >= 2M - 1 in shared memory: forward DIF
@@ -90,7 +99,8 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     const int tid = G::tid(), nthr = G::nthr();
     const BandRec br = a.bands[a.work[item / a.batch]];
     const int ch = item % a.batch;
-    const FftPlan &fp = a.ffts[br.fft];
+    __shared__ FftPlan plan_s;
+    const FftPlan &fp = WARP ? a.ffts[br.fft] : cta_plan(a.ffts[br.fft], plan_s, tid, nthr);
     float2 *buf = smem_band + (size_t)G::slot() * a.max_elems;
     const float2 *X = a.spec + (long long)ch * a.spec_pitch;
     const float *tab = a.table + br.tab_off;
@@ -159,7 +169,8 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     const int tid = G::tid(), nthr = G::nthr();
     const BandRec br = a.bands[a.work[item / a.batch]];
     const int ch = item % a.batch;
-    const FftPlan &fp = a.ffts[br.fft];
+    __shared__ FftPlan plan_s;
+    const FftPlan &fp = WARP ? a.ffts[br.fft] : cta_plan(a.ffts[br.fft], plan_s, tid, nthr);
     float2 *buf = smem_band + (size_t)G::slot() * a.max_elems;
     const int M = br.M;
     const float2 *in = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
