@@ -267,9 +267,13 @@ __device__ __forceinline__ bool dbg_ok(int *dbg, int site, long long idx, long l
 // COLFAST: consecutive threads take consecutive columns, else consecutive butterflies.
 template <int R, int SIGN, bool PAD, bool COLFAST, bool DIRECT, class Sync, class Load>
 __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
+    // plan fields are read once, ahead of the loops: the plan may sit in shared memory beside the data buffer,
+    // where the compiler must assume that a data store changes it
     const int s = fp.stride[0];
     const int total = s * t.ncols;
     const int spad = PAD ? s + fp.pad_delta : s;
+    const int logC = fp.logC;
+    const uint32_t smagic0 = fp.smagic[0];
     // every thread of the group runs every round: the first round contains the barrier that makes the
     // staged twiddle table visible, placed after the operand loads so both are in flight together
     for (int base = 0; base < total; base += nthr) {
@@ -279,7 +283,7 @@ __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, co
         if (active) {
             if (t.ncols == 1) { b = w; }
             else if (COLFAST) { b = fastdiv(w, t.ncols_magic, t.ncols); col = w - b * t.ncols; }
-            else { col = fastdiv(w, fp.smagic[0], s); b = w - col * s; }
+            else { col = fastdiv(w, smagic0, s); b = w - col * s; }
         }
         float re[R], im[R];
         if (active) {
@@ -293,7 +297,7 @@ __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, co
         if (base == 0) Sync::sync();
         if (active) {
             if (DIRECT) apply_twiddle_direct<R, SIGN>(tw, b, re, im);
-            else apply_twiddle_powers<R, SIGN>(tw, fp.logC, b, re, im);
+            else apply_twiddle_powers<R, SIGN>(tw, logC, b, re, im);
             float2 *p = t.buf + (b * (uint32_t)t.pitch + col);
             const uint32_t qstep = (uint32_t)spad * (uint32_t)t.pitch;
 #pragma unroll
@@ -309,13 +313,16 @@ __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, c
                                              int tid, int nthr) {
     const int s = fp.stride[j];
     const int total = (fp.M / R) * t.ncols;
+    const uint32_t smagic = fp.smagic[j], k1magic = fp.k1magic[j];
+    const int k1div = fp.k1div[j], logC = fp.logC;
+    const bool padded = PAD && fp.pad_delta != 0;
     for (int w = tid; w < total; w += nthr) {
         const uint32_t b = fastdiv(w, t.ncols_magic, t.ncols);
         const uint32_t col = w - b * t.ncols;
-        const uint32_t blk = fastdiv(b, fp.smagic[j], s);
+        const uint32_t blk = fastdiv(b, smagic, s);
         const uint32_t np = b - blk * s;
         uint32_t pos = blk * n_cur + np;
-        if (PAD) pos += fp.pad_delta ? fastdiv(blk, fp.k1magic[j], fp.k1div[j]) : 0u;
+        if (padded) pos += fastdiv(blk, k1magic, k1div);
         float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
         const uint32_t step = (uint32_t)s * (uint32_t)t.pitch;
         float re[R], im[R];
@@ -327,7 +334,7 @@ __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, c
         }
         if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
         if (DIRECT) { if (s > 1) apply_twiddle_direct<R, SIGN>(tw, np * tmul, re, im); }
-        else apply_twiddle_powers<R, SIGN>(tw, fp.logC, np * tmul, re, im);
+        else apply_twiddle_powers<R, SIGN>(tw, logC, np * tmul, re, im);
 #pragma unroll
         for (int q = 0; q < R; ++q) p[q * step] = make_float2(re[q], im[q]);
     }
@@ -341,6 +348,9 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
     const int nb = fp.M / R;
     const int total = nb * t.ncols;
     const int d = fp.nstages;
+    const bool padded = PAD && fp.pad_delta != 0;
+    const uint32_t k1magic = fp.k1magic[d - 1];
+    const int k1div = fp.k1div[d - 1];
     for (int w = tid; w < total; w += nthr) {
         uint32_t u, col;
         if (t.ncols == 1) { u = w; col = 0; }
@@ -371,7 +381,7 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
             }
         }
         uint32_t pos = b * R;
-        if (PAD) pos += fp.pad_delta ? fastdiv(b, fp.k1magic[d - 1], fp.k1div[d - 1]) : 0u;
+        if (padded) pos += fastdiv(b, k1magic, k1div);
         const float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
         float re[R], im[R];
         if (!CQT_CHK(t.dbg, 103, pos * t.pitch + col + (R - 1) * t.pitch, t.limit)) continue;
