@@ -160,6 +160,27 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     fft_fused<+1, Sync, false, true, false, true, false, false>(t, fp, tws, load, store, tid, nthr);
 }
 
+// Synthesis store of a regular band (all bins in range; plane row and table share the support index j = d - d0):
+// the window value is fetched ahead of the last butterfly, the product is stored after it.
+struct RegularStore {
+    const float *tab;
+    float2 *Ys;
+    int last_pos, first_neg, d0, shift_neg;
+    struct Fetched { float h; int j; };
+    __device__ __forceinline__ Fetched pre(int m, int) const {
+        const bool lo = m <= last_pos;
+        const bool ok = lo || m >= first_neg;
+        const int j = lo ? m - d0 : m - shift_neg;
+        Fetched f;
+        f.j = ok ? j : -1;
+        f.h = ok ? __ldg(tab + j) : 0.f;
+        return f;
+    }
+    __device__ __forceinline__ void operator()(int, int, float2 u, Fetched f) const {
+        if (f.j >= 0) Ys[f.j] = make_float2(f.h * u.x, f.h * u.y);
+    }
+};
+
 template <int THREADS, int MINB, bool WARP>
 __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
@@ -217,14 +238,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
         // regular band: all bins in range, plane row and table share the support index j = d - d0
         float2 *Ys = Y + (br.kc + br.d0);
         const int shift_neg = M + br.d0;
-        auto store_regular = [&](int m, int, float2 u) {
-            const bool lo = m <= last_pos;
-            if (!lo && m < first_neg) return;
-            const int j = lo ? m - br.d0 : m - shift_neg;
-            if (!CQT_CHK(a.dbg, 308, j, br.S)) return;
-            const float h = __ldg(tab + j);
-            Ys[j] = make_float2(h * u.x, h * u.y);
-        };
+        const RegularStore store_regular{tab, Ys, last_pos, first_neg, br.d0, shift_neg};
         auto load_regular = [&](int n, int) -> float2 { return __ldg(in + n); };
         fft_fused<-1, Sync, false, true, false, true, false, false>(t, fp, tws, load_regular, store_regular, tid, nthr);
         return;

@@ -3,6 +3,7 @@
 // Input in natural order, output in mixed-radix digit-reversed order (see FftPlan);
 // callers fold that permutation into their global-memory loads and stores.
 #pragma once
+#include <type_traits>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -340,6 +341,12 @@ __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, c
     }
 }
 
+// A store functor may split its work in two: pre(k, col), called before the butterfly's operands are read, fetches
+// whatever the store needs from global memory (a window value) so that the load's latency hides behind the
+// butterfly; operator()(k, col, value, fetched) then finishes.  Plain functors take (k, col, value).
+template <class Store>
+constexpr bool kStoreHasPre = !std::is_invocable<Store, int, int, float2>::value;
+
 // last stage (stride 1): operands from shared memory, result k of column col to store(k, col, value).
 // REV: thread index = low digits of k (consecutive threads store consecutive k), else thread index =
 // butterfly position.  COLFAST as above.
@@ -385,14 +392,28 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
         const float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
         float re[R], im[R];
         if (!CQT_CHK(t.dbg, 103, pos * t.pitch + col + (R - 1) * t.pitch, t.limit)) continue;
+        if constexpr (kStoreHasPre<Store>) {
+            decltype(store.pre(0, 0)) fetched[R];
 #pragma unroll
-        for (int q = 0; q < R; ++q) {
-            const float2 v = p[q * (uint32_t)t.pitch];
-            re[q] = v.x; im[q] = v.y;
+            for (int q = 0; q < R; ++q) fetched[q] = store.pre((int)(klow + q * nb), (int)col);
+#pragma unroll
+            for (int q = 0; q < R; ++q) {
+                const float2 v = p[q * (uint32_t)t.pitch];
+                re[q] = v.x; im[q] = v.y;
+            }
+            if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
+#pragma unroll
+            for (int q = 0; q < R; ++q) store((int)(klow + q * nb), (int)col, make_float2(re[q], im[q]), fetched[q]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < R; ++q) {
+                const float2 v = p[q * (uint32_t)t.pitch];
+                re[q] = v.x; im[q] = v.y;
+            }
+            if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
+#pragma unroll
+            for (int q = 0; q < R; ++q) store((int)(klow + q * nb), (int)col, make_float2(re[q], im[q]));
         }
-        if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
-#pragma unroll
-        for (int q = 0; q < R; ++q) store((int)(klow + q * nb), (int)col, make_float2(re[q], im[q]));
     }
 }
 
@@ -408,7 +429,10 @@ __device__ __forceinline__ void only_stage(const Tile &t, Load load, Store store
         }
         if (SIGN < 0) Codelet<R>::run(re, im); else Codelet<R>::run(im, re);
 #pragma unroll
-        for (int q = 0; q < R; ++q) store(q, col, make_float2(re[q], im[q]));
+        for (int q = 0; q < R; ++q) {
+            if constexpr (kStoreHasPre<Store>) store(q, col, make_float2(re[q], im[q]), store.pre(q, col));
+            else store(q, col, make_float2(re[q], im[q]));
+        }
     }
 }
 
