@@ -109,19 +109,18 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     const int first_neg = M + br.d0;          // slot of the most negative offset
     // slot m holds tab[d] X[kc + d] with d = m (m <= last_pos) or m - M (m >= first_neg), else zero
     auto load = [&](int m, int) -> float2 {
-        int d;
-        if (m <= last_pos) d = m;
-        else if (m >= first_neg) d = m - M;
-        else return make_float2(0.f, 0.f);
+        const bool lo = m <= last_pos;
+        if (!lo && m < first_neg) return make_float2(0.f, 0.f);
+        const int d = lo ? m : m - M;
         if (!CQT_CHK(a.dbg, 301, br.tab_off + (d - br.d0), a.table_len)) return make_float2(0.f, 0.f);
         const float g = __ldg(tab + (d - br.d0));
         const int k = br.kc + d;
-        if (!CQT_CHK(a.dbg, 302, k < 0 ? -k : (k > half ? a.N - k : k), half + 1)) return make_float2(0.f, 0.f);
-        float2 xv;
-        if (k < 0) xv = cconj(__ldg(X + (-k)));
-        else if (k > half) xv = cconj(__ldg(X + (a.N - k)));
-        else xv = __ldg(X + k);
-        return make_float2(g * xv.x, g * xv.y);
+        // bins outside 0..N/2 are the conjugates of their mirror bins
+        const bool mirrored = k < 0 || k > half;
+        const int km = k < 0 ? -k : (k > half ? a.N - k : k);
+        if (!CQT_CHK(a.dbg, 302, km, half + 1)) return make_float2(0.f, 0.f);
+        const float2 xv = __ldg(X + km);
+        return make_float2(g * xv.x, mirrored ? -(g * xv.y) : g * xv.y);
     };
     float2 *out = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
     if (fp.generic == 2) {
