@@ -23,7 +23,8 @@ Contents
   synthesise                                Eq. (synthesis)
   analyse_adjoint / synthesise_adjoint      real adjoints of Sec. 3.2
   pack / untangle / retangle                Eq. (pack), (untangle), (retangle)
-  slice_window / slicq_*                    sliced form (Sec. 4, slicing paragraph)
+  slice_window / slicq_*                    sliced form (Sec. 4, slicing paragraph); slicq_assemble lays the
+                                            sliced coefficients of each band on one time axis
 
 Parity status: every function here is pinned by tests/test_oracle_*.py against
 closed forms, brute-force sums, library routines or identities the paper
@@ -494,3 +495,24 @@ def slicq_overlap_add(y: np.ndarray, n_samples: int) -> np.ndarray:
     for s in range(ns):
         acc[..., s * H: s * H + sl] += y[..., s, :]
     return acc[..., H:H + n_samples]
+
+
+def slicq_assemble(lay: Layout, coeffs: Sequence[Sequence[np.ndarray]]) -> List[np.ndarray]:
+    """Re-assembly of sliced coefficients into one time series per band.
+
+    coeffs[i][band] holds the coefficients [..., M] of the i-th of n consecutive slices.  Slice i + 1 starts
+    sl/2 samples after slice i, i.e. M/2 coefficient periods later in a band of M coefficients, so band
+    lambda's series of length (n + 1) M/2 is the plain overlap-add out[i M/2 + m] += c_i[m].  (A layout of the
+    coefficients on a common time axis; sliced coefficients are not the whole-signal coefficients, Sec. 4.)"""
+    n = len(coeffs)
+    out = []
+    for b, band in enumerate(lay.bands):
+        M = band.M
+        if M % 2:
+            raise ValueError("band lengths must be even")
+        first = np.asarray(coeffs[0][b])
+        acc = np.zeros(first.shape[:-1] + ((n + 1) * (M // 2),), dtype=np.complex128)
+        for i in range(n):
+            acc[..., i * (M // 2): i * (M // 2) + M] += np.asarray(coeffs[i][b])
+        out.append(acc)
+    return out

@@ -50,3 +50,27 @@ def test_sliced_round_trip():
 def test_latency_is_one_slice():
     # one slice of 65,536 samples at 44.1 kHz (the figure quoted for the principal configuration)
     assert abs(65536 / 44100.0 * 1000.0 - 1486.1) < 0.05
+
+
+def test_assembled_band_series_places_every_coefficient_once():
+    """Re-assembly is a plain overlap-add at hop M/2: an impulse in coefficient m of slice i lands at i M/2 + m and
+    nowhere else; constants add to 1 + 1 where two slices overlap; the grand total is kept."""
+    lay = orc.build_layout(256.0, 6.0, 128.0, 6, 256, policy=orc.M_MULT4)
+    n = 4
+    rng = np.random.default_rng(3)
+    zero = [[np.zeros(b.M, dtype=np.complex128) for b in lay.bands] for _ in range(n)]
+    band, i, m = 5, 2, 3
+    zero[i][band][m] = 1.0 + 2.0j
+    out = orc.slicq_assemble(lay, zero)
+    M = lay.bands[band].M
+    assert out[band].shape[-1] == (n + 1) * M // 2
+    assert out[band][i * M // 2 + m] == 1.0 + 2.0j and np.count_nonzero(out[band]) == 1
+    assert all(np.count_nonzero(o) == 0 for j, o in enumerate(out) if j != band)
+    ones = [[np.ones(b.M, dtype=np.complex128) for b in lay.bands] for _ in range(n)]
+    for b, o in zip(lay.bands, orc.slicq_assemble(lay, ones)):
+        h = b.M // 2
+        assert np.all(o[:h] == 1) and np.all(o[h:n * h] == 2) and np.all(o[n * h:] == 1)
+    c = [[rng.standard_normal(b.M) + 1j * rng.standard_normal(b.M) for b in lay.bands] for _ in range(n)]
+    got = orc.slicq_assemble(lay, c)
+    for j in range(len(lay.bands)):
+        assert abs(got[j].sum() - sum(c[i][j].sum() for i in range(n))) < 1e-10
