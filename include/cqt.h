@@ -258,6 +258,34 @@ cqt_status slicq_reset(cqt_slicq *s);
 cqt_status slicq_destroy(cqt_slicq *s);
 size_t slicq_device_bytes(const cqt_slicq *s);
 
+/*
+ * Extras of the sliced form (the paper gives the slicing only; these make it usable for spectral processing).
+ *
+ * Processing between analysis and synthesis: the coefficients of an analysed slice (slicq_coeffs) may be edited
+ * in place, by kernels on the object's stream, until slicq_pull synthesises them.
+ *
+ * slicq_assemble lays the coefficients of n_slices consecutive analysed, not yet pulled slices
+ * first_slice .. first_slice + n_slices - 1 on one time axis per band: slice i + 1 starts sl/2 samples, i.e.
+ * M/2 coefficient periods of a band with M coefficients, after slice i, so band lambda's series has
+ * (n_slices + 1) M/2 entries, series[i M/2 + m] = sum over slices of c_i[m] (at most two terms, older slice
+ * first).  out (device): [channels][out_stride] complex64, band lambda's series starting at
+ * (n_slices + 1) * coeff_offset_lambda / 2; slicq_assembled_length = (n_slices + 1) * coeff_count / 2 entries per
+ * channel.  Entry t of a band's series belongs to stream time (first_slice - 1) sl/2 + t sl/M samples.  Sliced
+ * coefficients are not the coefficients of the whole signal (Sec. 4).  Errors: INVALID_ARG, STATE (a slice of the
+ * range is not held), CUDA.
+ *
+ * slicq_save_state / slicq_load_state copy the stream state (counters, input ring, overlap-add accumulator) to /
+ * from a host buffer of slicq_state_bytes, so that a stream can be suspended and resumed, also by another object
+ * created with the same plan shape, channels, transition and slices in flight (else CQT_ERR_STATE).  Saving needs
+ * every analysed slice to have been pulled (else CQT_ERR_STATE).  Both synchronise `stream`.
+ */
+int64_t slicq_assembled_length(const cqt_slicq *s, int64_t n_slices);
+cqt_status slicq_assemble(cqt_slicq *s, int64_t first_slice, int64_t n_slices, cqt_c64 *out, int64_t out_stride,
+                          void *stream);
+size_t slicq_state_bytes(const cqt_slicq *s);
+cqt_status slicq_save_state(cqt_slicq *s, void *host_buf, size_t bytes, void *stream);
+cqt_status slicq_load_state(cqt_slicq *s, const void *host_buf, size_t bytes, void *stream);
+
 const char *cqt_status_string(cqt_status status);
 
 #ifdef __cplusplus

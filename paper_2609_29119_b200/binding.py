@@ -74,6 +74,11 @@ EXPORTS = {
     "slicq_flush": (C.c_int, [C.c_void_p, C.c_void_p]),
     "slicq_reset": (C.c_int, [C.c_void_p]),
     "slicq_destroy": (C.c_int, [C.c_void_p]),
+    "slicq_assembled_length": (C.c_int64, [C.c_void_p, C.c_int64]),
+    "slicq_assemble": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]),
+    "slicq_state_bytes": (C.c_size_t, [C.c_void_p]),
+    "slicq_save_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "slicq_load_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "slicq_device_bytes": (C.c_size_t, [C.c_void_p]),
     "cqt_status_string": (C.c_char_p, [C.c_int]),
 }
@@ -323,6 +328,26 @@ class SliCQ:
 
     def reset(self) -> None:
         _check(self.lib.slicq_reset(self.handle), "slicq_reset")
+
+    def assemble(self, first_slice: int, n_slices: int, out=None, stream=None):
+        """slicq_assemble: [channels, (n_slices + 1) * coeff_count / 2] complex64, one time series per band."""
+        import torch
+        n = int(self.lib.slicq_assembled_length(self.handle, n_slices))
+        if out is None:
+            out = torch.empty((self.channels, n), dtype=torch.complex64, device=f"cuda:{self.plan.device}")
+        _check(self.lib.slicq_assemble(self.handle, first_slice, n_slices, out.data_ptr(), out.stride(0),
+                                       _stream_ptr(stream)), "slicq_assemble")
+        return out
+
+    def save_state(self, stream=None) -> bytes:
+        n = int(self.lib.slicq_state_bytes(self.handle))
+        buf = C.create_string_buffer(n)
+        _check(self.lib.slicq_save_state(self.handle, buf, n, _stream_ptr(stream)), "slicq_save_state")
+        return buf.raw
+
+    def load_state(self, state: bytes, stream=None) -> None:
+        buf = C.create_string_buffer(state, len(state))
+        _check(self.lib.slicq_load_state(self.handle, buf, len(state), _stream_ptr(stream)), "slicq_load_state")
 
 
 class _DeviceArray:

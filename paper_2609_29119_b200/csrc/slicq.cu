@@ -2,6 +2,7 @@
 // Tukey transition window, each analysed and synthesised independently, reconstructions
 // overlap-added in slice order.  All bookkeeping is host-side integer arithmetic; device work is
 // enqueued on the caller's stream and never synchronised here.
+#include <cstring>
 #include <algorithm>
 #include <cmath>
 #include <new>
@@ -21,6 +22,7 @@ struct cqt_slicq {
     cqt_c64 *d_coef = nullptr;           // [K][C][coeff_count]
     float *d_out = nullptr;              // [C][ring_out], output sample n at n mod ring_out
     void *d_ws = nullptr;
+    int *d_band_off = nullptr;           // [bands + 1] coefficient offsets of the bands, last = coeff_count
     size_t ws_bytes = 0, total_bytes = 0;
     int64_t n_in = 0;        // frames pushed
     int64_t next_slice = 0;  // first slice not yet analysed
@@ -69,6 +71,36 @@ __global__ void slicq_emit_kernel(const float *ring, long long R, long long pos,
     const int c = blockIdx.y;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         y[c * y_stride + i] = ring[c * R + (pos + i) % R];
+}
+
+// Re-assembly: band series of length (n + 1) M/2 per band, out[c][(n + 1) off/2 + t] = c_{i}[t - i M/2] + c_{i-1}[t - (i-1) M/2]
+// with i = floor(t / (M/2)) (terms whose slice index is outside 0..n-1 are absent), older slice first.
+// One thread per output; the band of an output follows from a binary search over the coefficient offsets.
+__global__ void slicq_assemble_kernel(const cqt_c64 *coef, long long cc, long long K, long long slot0, int C, long long n,
+                                      const int *band_off, int n_bands, cqt_c64 *out, long long out_stride) {
+    const int c = blockIdx.y;
+    const long long total = (n + 1) * (cc / 2);
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+        // band b: (n + 1) off_b / 2 <= e < (n + 1) off_{b+1} / 2
+        int lo = 0, hi = n_bands - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((n + 1) * (long long)(band_off[mid] / 2) <= e) lo = mid; else hi = mid - 1;
+        }
+        const long long off = band_off[lo], M = band_off[lo + 1] - off, h = M / 2;
+        const long long t = e - (n + 1) * (off / 2);
+        const long long i = t / h, m = t - i * h;
+        float re = 0.f, im = 0.f;
+        if (i >= 1) {   // second half of the older slice i - 1
+            const cqt_c64 v = coef[(((slot0 + i - 1) % K) * C + c) * cc + off + h + m];
+            re = v.re; im = v.im;
+        }
+        if (i < n) {    // first half of slice i
+            const cqt_c64 v = coef[(((slot0 + i) % K) * C + c) * cc + off + m];
+            re += v.re; im += v.im;
+        }
+        out[c * out_stride + e] = cqt_c64{re, im};
+    }
 }
 
 unsigned blocks_for(long long n) { return (unsigned)std::min<long long>(1024, std::max<long long>(1, (n + 255) / 256)); }
@@ -154,6 +186,14 @@ cqt_status slicq_create(const cqt_plan *plan, int channels, int64_t transition, 
     chk(cudaMalloc((void **)&s->d_coef, b_coef));
     chk(cudaMalloc((void **)&s->d_out, b_out));
     chk(cudaMalloc(&s->d_ws, s->ws_bytes));
+    {
+        const int64_t nb = cqt_plan_num_bands(plan);
+        std::vector<int> off((size_t)nb + 1);
+        for (int64_t b = 0; b < nb; ++b) off[(size_t)b] = (int)plan->lay.bands[(size_t)b].coeff_off;
+        off[(size_t)nb] = (int)cc;
+        chk(cudaMalloc((void **)&s->d_band_off, off.size() * sizeof(int)));
+        if (e == cudaSuccess) chk(cudaMemcpy(s->d_band_off, off.data(), off.size() * sizeof(int), cudaMemcpyHostToDevice));
+    }
     if (e == cudaSuccess) chk(cudaMemcpy(s->d_win, w.data(), b_win, cudaMemcpyHostToDevice));
     if (e == cudaSuccess) chk(cudaMemset(s->d_out, 0, b_out));
     s->total_bytes = b_win + b_in + b_stage + b_coef + b_out + s->ws_bytes;
@@ -238,12 +278,82 @@ cqt_status slicq_destroy(cqt_slicq *s) {
     int cur = 0;
     cudaGetDevice(&cur);
     cudaSetDevice(s->plan->device);
-    cudaFree(s->d_win); cudaFree(s->d_in); cudaFree(s->d_stage); cudaFree(s->d_coef); cudaFree(s->d_out); cudaFree(s->d_ws);
+    cudaFree(s->d_win); cudaFree(s->d_in); cudaFree(s->d_stage); cudaFree(s->d_coef); cudaFree(s->d_out); cudaFree(s->d_ws); cudaFree(s->d_band_off);
     cudaSetDevice(cur);
     delete s;
     return CQT_OK;
 }
 
 size_t slicq_device_bytes(const cqt_slicq *s) { return s ? s->total_bytes : 0; }
+
+int64_t slicq_assembled_length(const cqt_slicq *s, int64_t n_slices) {
+    if (!s || n_slices < 1) return 0;
+    return (n_slices + 1) * (cqt_plan_coeff_count(s->plan) / 2);
+}
+
+cqt_status slicq_assemble(cqt_slicq *s, int64_t first_slice, int64_t n_slices, cqt_c64 *out, int64_t out_stride, void *stream) {
+    if (!s || !out || n_slices < 1 || first_slice < 0) return CQT_ERR_INVALID_ARG;
+    if (out_stride < slicq_assembled_length(s, n_slices)) return CQT_ERR_INVALID_ARG;
+    if (first_slice < s->next_synth || first_slice + n_slices > s->next_slice) return CQT_ERR_STATE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int64_t cc = cqt_plan_coeff_count(s->plan);
+    dim3 grid(blocks_for((n_slices + 1) * (cc / 2)), (unsigned)s->C);
+    slicq_assemble_kernel<<<grid, 256, 0, st>>>(s->d_coef, cc, s->K, first_slice % s->K, s->C, n_slices, s->d_band_off,
+                                                (int)cqt_plan_num_bands(s->plan), out, out_stride);
+    return cudaGetLastError() == cudaSuccess ? CQT_OK : CQT_ERR_CUDA;
+}
+
+// Saved state: header, then the input ring and the output ring ([C][ring] floats each).
+struct SlicqStateHeader {
+    uint32_t magic, version;
+    int32_t channels;
+    int32_t pad_;
+    int64_t sl, tr, K, ring_in, ring_out, coeff_count;
+    int64_t n_in, next_slice, next_synth, n_out;
+};
+static const uint32_t kStateMagic = 0x51436c53u;   // "SlCQ"
+
+size_t slicq_state_bytes(const cqt_slicq *s) {
+    if (!s) return 0;
+    return sizeof(SlicqStateHeader) + (size_t)s->C * (size_t)(s->ring_in + s->ring_out) * sizeof(float);
+}
+
+cqt_status slicq_save_state(cqt_slicq *s, void *host_buf, size_t bytes, void *stream) {
+    if (!s || !host_buf) return CQT_ERR_INVALID_ARG;
+    if (bytes < slicq_state_bytes(s)) return CQT_ERR_WORKSPACE;
+    if (s->next_synth != s->next_slice) return CQT_ERR_STATE;    // analysed slices await slicq_pull
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    SlicqStateHeader h{kStateMagic, 1u, s->C, 0, s->sl, s->tr, s->K, s->ring_in, s->ring_out, cqt_plan_coeff_count(s->plan),
+                       s->n_in, s->next_slice, s->next_synth, s->n_out};
+    char *p = static_cast<char *>(host_buf);
+    std::memcpy(p, &h, sizeof h);
+    const size_t b_in = (size_t)s->C * s->ring_in * sizeof(float), b_out = (size_t)s->C * s->ring_out * sizeof(float);
+    cudaError_t e = cudaMemcpyAsync(p + sizeof h, s->d_in, b_in, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(p + sizeof h + b_in, s->d_out, b_out, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? CQT_OK : CQT_ERR_CUDA;
+}
+
+cqt_status slicq_load_state(cqt_slicq *s, const void *host_buf, size_t bytes, void *stream) {
+    if (!s || !host_buf) return CQT_ERR_INVALID_ARG;
+    if (bytes < sizeof(SlicqStateHeader)) return CQT_ERR_INVALID_ARG;
+    SlicqStateHeader h;
+    std::memcpy(&h, host_buf, sizeof h);
+    if (h.magic != kStateMagic || h.version != 1u) return CQT_ERR_INVALID_ARG;
+    if (h.channels != s->C || h.sl != s->sl || h.tr != s->tr || h.K != s->K || h.ring_in != s->ring_in ||
+        h.ring_out != s->ring_out || h.coeff_count != cqt_plan_coeff_count(s->plan))
+        return CQT_ERR_STATE;                                     // saved by an object of another shape
+    if (bytes < slicq_state_bytes(s)) return CQT_ERR_INVALID_ARG;
+    if (h.next_synth != h.next_slice || h.n_in < 0 || h.n_out < 0 || h.n_out > h.n_in) return CQT_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const char *p = static_cast<const char *>(host_buf);
+    const size_t b_in = (size_t)s->C * s->ring_in * sizeof(float), b_out = (size_t)s->C * s->ring_out * sizeof(float);
+    cudaError_t e = cudaMemcpyAsync(s->d_in, p + sizeof h, b_in, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s->d_out, p + sizeof h + b_in, b_out, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);          // the host buffer may be pageable and reused
+    if (e != cudaSuccess) return CQT_ERR_CUDA;
+    s->n_in = h.n_in; s->next_slice = h.next_slice; s->next_synth = h.next_synth; s->n_out = h.n_out;
+    return CQT_OK;
+}
 
 }  // extern "C"

@@ -96,3 +96,115 @@ def test_push_beyond_the_slots_in_flight_is_refused():
     assert sq.push(x[:, :H]) == 1
     sq.close()
     plan.close()
+
+
+def test_assembled_coefficients_match_oracle():
+    """slicq_assemble against the oracle's overlap-add of the oracle's own per-slice coefficients."""
+    from paper_2609_29119_b200 import CqtError, SliCQ
+    lay, plan = oracle_layout(W), library_plan(W)
+    x = wl.make_signal(W)
+    H = W.slice_len // 2
+    sq = SliCQ(plan, x.shape[0], W.transition, 6)
+    xd = torch.from_numpy(x).cuda()
+    assert sq.push(xd[:, :5 * H]) == 5
+    slices = orc.slicq_cut(x.astype(np.float64), W.slice_len, W.transition)
+    for first, n in ((0, 5), (1, 3), (4, 1)):
+        got = sq.assemble(first, n).cpu().numpy()
+        want = orc.slicq_assemble(lay, [orc.analyse(lay, slices[:, s, :]) for s in range(first, first + n)])
+        assert got.shape[1] == (n + 1) * lay.coeff_count // 2
+        o = 0
+        for b, wb in zip(lay.bands, want):
+            g = got[:, o:o + wb.shape[-1]]
+            assert np.linalg.norm(g - wb) <= 1e-5 * np.linalg.norm(wb), (first, n, b.kc)
+            o += wb.shape[-1]
+    with pytest.raises(CqtError) as e:
+        sq.assemble(3, 3)             # slice 5 has not been analysed
+    assert e.value.status == -6
+    sq.close()
+    plan.close()
+
+
+def test_coefficients_edited_between_push_and_pull_are_what_is_synthesised():
+    """Processing hook: zero all bands above one index in every slice before pulling; the output is the oracle's
+    overlap-add of the slices synthesised from the same edited coefficients."""
+    from paper_2609_29119_b200 import SliCQ
+    lay, plan = oracle_layout(W), library_plan(W)
+    x = wl.make_signal(W)
+    n, H = x.shape[1], W.slice_len // 2
+    keep = lay.coeff_offsets[len(lay.bands) // 2]        # coefficients of the lower half of the bands
+    sq = SliCQ(plan, x.shape[0], W.transition, 4)
+    xd = torch.from_numpy(x).cuda()
+    out = torch.zeros((x.shape[0], n + 2 * W.slice_len), device="cuda")
+    got = pos = done = 0
+    while pos < n:
+        m = min(H, n - pos)
+        now = sq.push(xd[:, pos:pos + m])
+        for s in range(done, now):
+            sq.coeffs(s)[:, keep:] = 0
+        done = now
+        pos += m
+        got += sq.pull(out[:, got:])
+    before = sq.push(xd[:, :0])
+    sq.flush()
+    for s in range(before, sq.push(xd[:, :0])):
+        sq.coeffs(s)[:, keep:] = 0
+    got += sq.pull(out[:, got:])
+    slices = orc.slicq_cut(x.astype(np.float64), W.slice_len, W.transition)
+    rec = []
+    for s in range(slices.shape[1]):
+        c = orc.analyse(lay, slices[:, s, :])
+        c = [cb if i < len(lay.bands) // 2 else np.zeros_like(cb) for i, cb in enumerate(c)]
+        rec.append(orc.synthesise(lay, c))
+    want = orc.slicq_overlap_add(np.stack(rec, axis=1), n)
+    y = out[:, :n].cpu().numpy()
+    rel = np.linalg.norm(y - want, axis=-1) / np.linalg.norm(want, axis=-1)
+    assert rel.max() <= 1e-5, rel
+    assert snr_db(x, y).max() < 30.0          # and it is not the identity any more
+    sq.close()
+    plan.close()
+
+
+def test_saved_state_resumes_the_stream_bit_for_bit():
+    from paper_2609_29119_b200 import CqtError, SliCQ
+    plan = library_plan(W)
+    x = wl.make_signal(W)
+    n, H = x.shape[1], W.slice_len // 2
+    xd = torch.from_numpy(x).cuda()
+
+    def run(sq, lo, hi, out, got):
+        pos = lo
+        while pos < hi:
+            m = min(H + 37, hi - pos)
+            sq.push(xd[:, pos:pos + m])
+            pos += m
+            got += sq.pull(out[:, got:])
+        return got
+    ref = torch.zeros((x.shape[0], n + 2 * W.slice_len), device="cuda")
+    a = SliCQ(plan, x.shape[0], W.transition, 4)
+    g = run(a, 0, n, ref, 0)
+    a.flush()
+    g += a.pull(ref[:, g:])
+    cut = 2 * H + 301
+    out = torch.zeros_like(ref)
+    b = SliCQ(plan, x.shape[0], W.transition, 4)
+    gb = run(b, 0, cut, out, 0)
+    b.push(xd[:, cut:cut + H])               # leaves an analysed slice waiting: saving is refused
+    with pytest.raises(CqtError) as e:
+        b.save_state()
+    assert e.value.status == -6
+    gb += b.pull(out[:, gb:])
+    state = b.save_state()
+    b.close()
+    c = SliCQ(plan, x.shape[0], W.transition, 4)
+    c.load_state(state)
+    gc = run(c, cut + H, n, out, gb)
+    c.flush()
+    gc += c.pull(out[:, gc:])
+    assert gc == g
+    assert torch.equal(out[:, :g], ref[:, :g])
+    other = SliCQ(plan, x.shape[0], W.transition, 3)
+    with pytest.raises(CqtError) as e:
+        other.load_state(state)              # saved by an object with another number of slices in flight
+    assert e.value.status == -6
+    other.close(); c.close(); a.close()
+    plan.close()
