@@ -247,20 +247,39 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
 
 // ---------------------------------------------------------------- inverse: overlap-add + retangle
 // sum over the bands covering bin k, in band order
-__device__ __forceinline__ float2 gather_bin(const LongArgs &a, const float2 *__restrict__ Y, int k) {
-    if (!CQT_CHK(a.dbg, 205, k, a.Lp + 1)) return make_float2(0.f, 0.f);
-    const int32_t cv = __ldg(a.cover + k);     // (plane of the first covering band << 8) | number of covering bands
-    const int n = cv & 255;
-    if (!CQT_CHK(a.dbg, 206, n, a.planes + 1)) return make_float2(0.f, 0.f);
-    const int plane_len = (int)a.y_plane, wrap = a.planes * plane_len;
-    int off = (cv >> 8) * plane_len + k;
+// Sum over the bands covering bin k, in band order.  The cover word is (plane of the first covering band << 8) | number
+// of covering bands; band i of the range sits in plane (first + i) mod planes.  The first kUnroll plane values are loaded
+// unconditionally-predicated before any is used, so that their latencies overlap; absent terms add +0.
+constexpr int kGatherUnroll = 4;
+struct GatherLoads {
+    float2 v[kGatherUnroll];
+    int n, off, plane_len, wrap;
+};
+__device__ __forceinline__ GatherLoads gather_issue(const LongArgs &a, const float2 *__restrict__ Y, int k, int32_t cv) {
+    GatherLoads g;
+    g.n = cv & 255;
+    g.plane_len = (int)a.y_plane;
+    g.wrap = a.planes * g.plane_len;
+    g.off = (cv >> 8) * g.plane_len + k;
+    if (!CQT_CHK(a.dbg, 206, g.n, a.planes + 1)) g.n = 0;
+#pragma unroll
+    for (int i = 0; i < kGatherUnroll; ++i) {
+        g.v[i] = i < g.n ? __ldg(Y + g.off) : make_float2(0.f, 0.f);
+        g.off += g.plane_len;
+        if (g.off >= g.wrap) g.off -= g.wrap;
+    }
+    return g;
+}
+__device__ __forceinline__ float2 gather_finish(const float2 *__restrict__ Y, GatherLoads &g) {
     float2 acc = make_float2(0.f, 0.f);
-    for (int i = 0; i < n; ++i) {
-        const float2 v = __ldg(Y + off);
+#pragma unroll
+    for (int i = 0; i < kGatherUnroll; ++i) { acc.x += g.v[i].x; acc.y += g.v[i].y; }
+    for (int i = kGatherUnroll; i < g.n; ++i) {
+        const float2 v = __ldg(Y + g.off);
         acc.x += v.x;
         acc.y += v.y;
-        off += plane_len;
-        if (off >= wrap) off -= wrap;
+        g.off += g.plane_len;
+        if (g.off >= g.wrap) g.off -= g.wrap;
     }
     return acc;
 }
@@ -277,8 +296,11 @@ __global__ void __launch_bounds__(256) gather_retangle_kernel(LongArgs a) {
     const float2 *Y = a.Y + (long long)ch * a.y_pitch;
     float2 *Z = a.Z + (long long)ch * a.t_pitch;
     const int m = Lp - q;
-    float2 xq = gather_bin(a, Y, q);
-    float2 xm = gather_bin(a, Y, m);
+    if (!CQT_CHK(a.dbg, 205, m, Lp + 1)) return;
+    const int32_t cvq = __ldg(a.cover + q), cvm = __ldg(a.cover + m);
+    GatherLoads gq = gather_issue(a, Y, q, cvq), gm = gather_issue(a, Y, m, cvm);
+    float2 xq = gather_finish(Y, gq);
+    float2 xm = gather_finish(Y, gm);
     if (q == 0) { xq.y = 0.f; xm.y = 0.f; }   // bins 0 and N/2 are made real
     const float2 w = twiddle(a.tw + a.tw_n, a.log_n_c, (uint32_t)q);
     {
