@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
 // Sum over the bands covering bin k, in band order.  The cover word is (plane of the first covering band << 8) | number
 // of covering bands; band i of the range sits in plane (first + i) mod planes.  The first kUnroll plane values are loaded
 // unconditionally-predicated before any is used, so that their latencies overlap; absent terms add +0.
-constexpr int kGatherUnroll = 4;
+constexpr int kGatherUnroll = 3;
 struct GatherLoads {
     float2 v[kGatherUnroll];
     int n, off, plane_len, wrap;
@@ -288,7 +288,7 @@ __device__ __forceinline__ float2 gather_finish(const float2 *__restrict__ Y, Ga
 // packed bins of the pair follow from the same two values (Eq. retangle with w_{Lp-q} = -conj w_q):
 //   Z_q      = s [ (X_q + conj X_m) + i conj(w) (X_q - conj X_m) ]
 //   Z_{Lp-q} = s [ (X_m + conj X_q) - i w (X_m - conj X_q) ],   m = Lp - q, w = exp(-2 pi i q / N), s = 1/(2 Lp)
-__global__ void __launch_bounds__(256) gather_retangle_kernel(LongArgs a) {
+__global__ void __launch_bounds__(256, 8) gather_retangle_kernel(LongArgs a) {
     const int ch = blockIdx.y;
     const int Lp = a.Lp;
     const int q = blockIdx.x * blockDim.x + threadIdx.x;
