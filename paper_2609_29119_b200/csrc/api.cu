@@ -183,7 +183,7 @@ void free_device(cqt_plan *p) {
     int cur = 0;
     cudaGetDevice(&cur);
     cudaSetDevice(p->device);
-    cudaFree(p->d.bands); cudaFree(p->d.ffts); cudaFree(p->d.tw);
+    cudaFree(p->d.bands); cudaFree(p->d.items); cudaFree(p->d.ffts); cudaFree(p->d.tw);
     cudaFree(p->d.tab_analysis); cudaFree(p->d.tab_synthesis);
     cudaFree(p->d.tab_analysis_adj); cudaFree(p->d.tab_synthesis_adj);
     cudaFree(p->d.cover); cudaFree(p->d.dbg); cudaFree(p->d.zero_seg);
@@ -491,6 +491,15 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
     cudaError_t e = cudaSuccess;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
     chk(upload(p->d.bands, p->bands));
+    {
+        std::vector<BandItem> items(p->bands.size());
+        for (size_t i = 0; i < items.size(); ++i) {
+            items[i].br = p->bands[i];
+            if (p->bands[i].fft >= 0) items[i].fp = p->ffts[(size_t)p->bands[i].fft];
+            else std::memset(&items[i].fp, 0, sizeof(FftPlan));
+        }
+        chk(upload(p->d.items, items));
+    }
     chk(upload(p->d.ffts, p->ffts));
     chk(upload(p->d.tw, tw));
     chk(upload(p->d.tab_analysis, tA));

@@ -14,7 +14,7 @@
 namespace cqt {
 
 struct BandArgs {
-    const BandRec *bands;
+    const BandItem *items;   // per band: record + radix plan
     const FftPlan *ffts;
     const float2 *tw;
     const float *table;
@@ -45,13 +45,14 @@ struct Group {
 
 extern __shared__ float2 smem_band[];
 
-// One-CTA-per-item kernels keep the item's radix plan in shared memory: its fields are read inside the stage
-// loops, and a shared-memory copy costs a short-latency load where the global original costs a cache lookup.
-__device__ __forceinline__ const FftPlan &cta_plan(const FftPlan &g, FftPlan &s, int tid, int nthr) {
-    constexpr int kWords = (int)(sizeof(FftPlan) / sizeof(int));
+// The work item's band record and radix plan are fetched together, once, into shared memory: their fields are
+// read inside the stage loops, where a shared-memory copy costs a short-latency load and the global original a
+// cache lookup, and one cooperative load replaces a chain of two dependent ones.
+template <class Sync>
+__device__ __forceinline__ void fetch_item(const BandItem &g, BandItem &s, int tid, int nthr) {
+    constexpr int kWords = (int)(sizeof(BandItem) / sizeof(int));
     for (int i = tid; i < kWords; i += nthr) reinterpret_cast<int *>(&s)[i] = __ldg(reinterpret_cast<const int *>(&g) + i);
-    __syncthreads();
-    return s;
+    Sync::sync();
 }
 
 // Chirp-z (Bluestein) evaluation of an M-point DFT of sign SIGN whose length has a large prime factor:
@@ -97,10 +98,12 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     const int item = G::item();
     if (item >= a.n_work * a.batch) return;   // whole group exits together
     const int tid = G::tid(), nthr = G::nthr();
-    const BandRec br = a.bands[a.work[item / a.batch]];
+    __shared__ BandItem item_s[WARP ? 8 : 1];
+    BandItem &it = item_s[G::slot()];
+    fetch_item<Sync>(a.items[a.work[item / a.batch]], it, tid, nthr);
+    const BandRec br = it.br;
     const int ch = item % a.batch;
-    __shared__ FftPlan plan_s;
-    const FftPlan &fp = WARP ? a.ffts[br.fft] : cta_plan(a.ffts[br.fft], plan_s, tid, nthr);
+    const FftPlan &fp = it.fp;
     float2 *buf = smem_band + (size_t)G::slot() * a.max_elems;
     const float2 *X = a.spec + (long long)ch * a.spec_pitch;
     const float *tab = a.table + br.tab_off;
@@ -187,10 +190,12 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     const int item = G::item();
     if (item >= a.n_work * a.batch) return;
     const int tid = G::tid(), nthr = G::nthr();
-    const BandRec br = a.bands[a.work[item / a.batch]];
+    __shared__ BandItem item_s[WARP ? 8 : 1];
+    BandItem &it = item_s[G::slot()];
+    fetch_item<Sync>(a.items[a.work[item / a.batch]], it, tid, nthr);
+    const BandRec br = it.br;
     const int ch = item % a.batch;
-    __shared__ FftPlan plan_s;
-    const FftPlan &fp = WARP ? a.ffts[br.fft] : cta_plan(a.ffts[br.fft], plan_s, tid, nthr);
+    const FftPlan &fp = it.fp;
     float2 *buf = smem_band + (size_t)G::slot() * a.max_elems;
     const int M = br.M;
     const float2 *in = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
@@ -247,7 +252,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
 
 static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *table, int64_t batch) {
     BandArgs a{};
-    a.bands = p.d.bands;
+    a.items = p.d.items;
     a.ffts = p.d.ffts;
     a.tw = p.d.tw;
     a.table = table;

@@ -47,6 +47,7 @@ struct TwoPassGroup {
 
 struct DevicePlan {
     BandRec *bands = nullptr;
+    BandItem *items = nullptr;         // per band: record + plan (plan zeroed for bands on the two-pass kernels)
     FftPlan *ffts = nullptr;
     float2 *tw = nullptr;
     float *tab_analysis = nullptr;     // g / M

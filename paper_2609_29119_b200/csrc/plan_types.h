@@ -49,6 +49,13 @@ struct BandRec {
     int32_t pad_[2];
 };
 
+// A band record together with the radix plan of its length: what one work item of the band kernels needs,
+// fetched in one cooperative load.
+struct BandItem {
+    BandRec br;
+    FftPlan fp;
+};
+
 // A band transformed in two passes (M = A * B) through a scratch row.
 struct TwoPassRec {
     int32_t band;
