@@ -91,6 +91,7 @@ __device__ __forceinline__ void stage_table(float2 *dst, const float2 *__restric
 // Every pass exists once as a template over a compile-time Shape (radices, columns, pitch) and is instantiated
 // for the common shapes plus the run-time planned fallback; the kernels pick the instantiation that matches.
 using DynShape = Shape<0, 0, 0, 0, 0>;
+using Sh_16_16_8_8_9 = Shape<16, 16, 8, 8, 9>;
 using Sh_8_8_8_16_16 = Shape<8, 8, 8, 16, 16>;
 using Sh_16_16_1_16_16 = Shape<16, 16, 1, 16, 16>;
 using Sh_16_8_1_16_16 = Shape<16, 8, 1, 16, 16>;
@@ -342,12 +343,16 @@ __device__ __forceinline__ void rows_inv_body(const LongArgs &a, const FftPlan &
         for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[SH::pos(fp, (uint32_t)j)], a.valid_len, a.aligned);
     } else {
         float2 *T = a.T + (long long)ch * a.t_pitch;
+        // The inverse keeps its intermediate transposed, Tinv[j2][q1]: consecutive threads take consecutive rows r, so
+        // the shared-memory reads (odd pitch) are conflict-free and the 8-byte stores of a warp fall in runs of TW rows;
+        // reading the digit-reversed positions of consecutive j2 instead would hit one bank 16 times.
+        const int log_tw = 31 - __clz(TW);
         for (int e = tid; e < ncols * B; e += nthr) {
-            const int r = e >> a.log_b, j2 = e - (r << a.log_b);
+            const int j2 = e >> log_tw, r = e - (j2 << log_tw);
             const int q1 = t * TW + r;
             const float2 v = buf[SH::pos(fp, (uint32_t)j2) * (uint32_t)pitch + r];
             const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
-            if (CQT_CHK(a.dbg, 207, q1 * B + j2, a.Lp)) T[q1 * B + j2] = cmul(v, w);
+            if (CQT_CHK(a.dbg, 207, j2 * A + q1, a.Lp)) T[j2 * A + q1] = cmul(v, w);
         }
     }
 }
@@ -380,16 +385,17 @@ __device__ __forceinline__ void cols_inv_body(const LongArgs &a, const FftPlan &
     const int TW = a.tw_cols;
     const float2 *T = a.T + (long long)ch * a.t_pitch;
     float *row = a.x_out + (long long)ch * a.x_stride;
+    // Tinv[j2][q1]: a column of the tile is a contiguous run of A values, so consecutive threads take consecutive q1
     auto load = [&](int q1, int c) -> float2 {
-        const int i = q1 * a.B + j2_0 + c;
+        const int i = (j2_0 + c) * a.A + q1;
         return CQT_CHK(a.dbg, 208, i, a.Lp) ? __ldg(T + i) : make_float2(0.f, 0.f);
     };
     auto store = [&](int j1, int c, float2 v) { store_packed(row, j1 * a.B + j2_0 + c, v, a.valid_len, a.aligned); };
     if constexpr (SH::is_static) {
-        tile_fft_static<SH, +1, true, false>(buf, tws, load, store, tid, nthr);
+        tile_fft_static<SH, +1, false, false>(buf, tws, load, store, tid, nthr);
     } else {
-        const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
-        fft_fused<+1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+        const Tile t{buf, TW | 1, TW, a.cols_magic, a.A * (TW | 1), a.dbg};
+        fft_fused<+1, BlockSync, true, false, false, false, true, true>(t, fp, tws, load, store, tid, nthr);
     }
 }
 
@@ -400,15 +406,15 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     const int ch = blockIdx.y;
     const FftPlan &fp = a.ffts[a.fft_A];
     float2 *buf = smem_long;
-    float2 *tws = buf + (size_t)a.A * TW;
+    float2 *tws = buf + (size_t)a.A * (TW | 1);
     stage_full(tws, a.tw, fp, tid, nthr);
 #undef CQT_SHAPE_LIST
 #define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_16, __VA_ARGS__)          \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_16, __VA_ARGS__)        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_16, __VA_ARGS__)         \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_8, __VA_ARGS__)           \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_8_8_8, __VA_ARGS__)
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_17, __VA_ARGS__)          \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_17, __VA_ARGS__)        \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_17, __VA_ARGS__)         \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_9, __VA_ARGS__)           \
+    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_8_8_9, __VA_ARGS__)
     CQT_DISPATCH_SHAPES(cols_inv_body, fp, TW, a, fp, buf, tws, j2_0, ch, tid, nthr);
 }
 #undef CQT_SHAPE_LIST
@@ -465,7 +471,7 @@ static size_t rows_inv_smem(const cqt_plan &p) {
 }
 static size_t cols_smem(const cqt_plan &p) {
     const LongFft &lf = p.lf;
-    return ((size_t)lf.A * lf.tw_cols + plan_tw(p, lf.fft_A) + lf.n_lp) * 8;
+    return ((size_t)lf.A * (lf.tw_cols | 1) + plan_tw(p, lf.fft_A) + lf.n_lp) * 8;   // odd pitch in the inverse pass
 }
 
 static int threads_for(size_t butterflies) {
