@@ -352,6 +352,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
         p->cls[c].threads = threads[c];
         p->cls[c].min_blocks = minb[c];
         p->cls[c].items_per_cta = c == 0 ? 8 : 1;
+        p->cls[c].max_radix = c <= 1 ? 8 : (c == 2 ? 12 : 16);
     }
     std::vector<int> order(L.bands.size());
     for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
@@ -392,7 +393,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
         int64_t A2 = 0;
         if (!single) { A2 = split_two_pass(M); single = A2 == 0; }
         if (single) {
-            g_radix_cap = c <= 1 ? 8 : (c == 2 ? 12 : 16);   // short bands: fewer registers, more CTAs per SM
+            g_radix_cap = p->cls[c].max_radix;   // short bands: fewer registers, more CTAs per SM
             p->bands[i].fft = plan_for(M, false);
             g_radix_cap = 16;
             if (p->bands[i].fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }

@@ -91,7 +91,7 @@ __device__ __forceinline__ void chirp_z_transform(float2 *buf, const FftPlan &fp
     }
 }
 
-template <int THREADS, int MINB, bool WARP>
+template <int THREADS, int MINB, bool WARP, int MAXR>
 __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
     using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
@@ -156,10 +156,10 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
             const float2 xv = __ldg(Xs + j);
             return make_float2(g * xv.x, g * xv.y);
         };
-        fft_fused<+1, Sync, false, true, false, true, false, false>(t, fp, tws, load_regular, store, tid, nthr);
+        fft_fused<+1, Sync, false, true, false, true, false, false, MAXR>(t, fp, tws, load_regular, store, tid, nthr);
         return;
     }
-    fft_fused<+1, Sync, false, true, false, true, false, false>(t, fp, tws, load, store, tid, nthr);
+    fft_fused<+1, Sync, false, true, false, true, false, false, MAXR>(t, fp, tws, load, store, tid, nthr);
 }
 
 // Synthesis store of a regular band (all bins in range; plane row and table share the support index j = d - d0):
@@ -183,7 +183,7 @@ struct RegularStore {
     }
 };
 
-template <int THREADS, int MINB, bool WARP>
+template <int THREADS, int MINB, bool WARP, int MAXR>
 __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
     using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
@@ -244,10 +244,10 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
         const int shift_neg = M + br.d0;
         const RegularStore store_regular{tab, Ys, last_pos, first_neg, br.d0, shift_neg};
         auto load_regular = [&](int n, int) -> float2 { return __ldg(in + n); };
-        fft_fused<-1, Sync, false, true, false, true, false, false>(t, fp, tws, load_regular, store_regular, tid, nthr);
+        fft_fused<-1, Sync, false, true, false, true, false, false, MAXR>(t, fp, tws, load_regular, store_regular, tid, nthr);
         return;
     }
-    fft_fused<-1, Sync, false, true, false, true, false, false>(t, fp, tws, load, store, tid, nthr);
+    fft_fused<-1, Sync, false, true, false, true, false, false, MAXR>(t, fp, tws, load, store, tid, nthr);
 }
 
 static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *table, int64_t batch) {
@@ -268,15 +268,17 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
     return a;
 }
 
-// kernel instantiations: (threads per CTA, CTAs per SM the registers must allow, one warp per item)
+// kernel instantiations: (threads per CTA, CTAs per SM the registers must allow, one warp per item, largest radix
+// compiled in).  The first five are the default classes; the last two serve the class-tuning environment hooks.
 #define CQT_KERNEL_TABLE(X) \
-    X(256, 4, true) X(64, 16, false) X(256, 4, false) X(512, 2, false) X(1024, 1, false) X(128, 8, false) X(256, 2, false)
+    X(256, 4, true, 8) X(64, 16, false, 8) X(256, 4, false, 12) X(512, 2, false, 16) X(1024, 1, false, 16) \
+    X(128, 8, false, 16) X(256, 2, false, 16)
 
 template <bool ANALYSIS>
 static const void *class_kernel(const BandClass &c) {
-#define X(T, B, W)                                                   \
-    if (c.threads == T && c.min_blocks == B && (c.items_per_cta > 1) == W) \
-        return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W> : (const void *)bands_to_spectrum_kernel<T, B, W>;
+#define X(T, B, W, R)                                                                        \
+    if (c.threads == T && c.min_blocks == B && (c.items_per_cta > 1) == W && c.max_radix <= R) \
+        return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W, R> : (const void *)bands_to_spectrum_kernel<T, B, W, R>;
     CQT_KERNEL_TABLE(X)
 #undef X
     return nullptr;

@@ -490,21 +490,23 @@ __device__ void fft_dit_inverse(const Tile &t, const FftPlan &fp, const float2 *
 
 // Runs the first `nrun` stages of the plan (nrun = nstages: the whole transform with the last stage fused
 // into `store`; nrun = nstages - 1... not offered: use fft_fused_keep for "results stay in shared memory").
+// MAXR: largest radix the plan may contain (larger cases are not compiled; the plan builder caps the radices of
+// short bands, whose kernels need neither the code nor the registers of the big codelets).
 // Requires a non-generic plan.  tw = shared-memory copy of the plan's two-level table, written by the
 // caller (stage_twiddles) WITHOUT a barrier after it: the first stage synchronises once its operand loads
 // are issued.  The routine synchronises between stages, not at the end.
-template <int SIGN, class Sync, bool POW2, bool PAD, bool COLFAST_IN, bool REV, bool COLFAST_OUT, bool DIRECT, class Load, class Store>
+template <int SIGN, class Sync, bool POW2, bool PAD, bool COLFAST_IN, bool REV, bool COLFAST_OUT, bool DIRECT, int MAXR = 16, class Load, class Store>
 __device__ __forceinline__ void fft_fused(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, Store store, int tid, int nthr) {
     const int d = fp.nstages;
     if (d == 1) {
         Sync::sync();   // tables staged by the caller become visible to the functors
-#define X(RR) case RR: only_stage<RR, SIGN>(t, load, store, tid, nthr); break;
+#define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) only_stage<RR, SIGN>(t, load, store, tid, nthr); break;
         if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
         else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
         return;
     }
-#define X(RR) case RR: first_stage<RR, SIGN, PAD, COLFAST_IN, DIRECT, Sync>(t, fp, tw, load, tid, nthr); break;
+#define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) first_stage<RR, SIGN, PAD, COLFAST_IN, DIRECT, Sync>(t, fp, tw, load, tid, nthr); break;
     if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
     else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
@@ -512,7 +514,7 @@ __device__ __forceinline__ void fft_fused(const Tile &t, const FftPlan &fp, cons
     int n_cur = fp.stride[0], tmul = fp.radix[0];
 #pragma unroll 1
     for (int j = 1; j < d - 1; ++j) {
-#define X(RR) case RR: middle_stage<RR, SIGN, PAD, DIRECT>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
+#define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) middle_stage<RR, SIGN, PAD, DIRECT>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
         if (POW2) { switch (fp.radix[j]) { CQT_RADIX_CASES_POW2(X) default: break; } }
         else { switch (fp.radix[j]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
@@ -520,7 +522,7 @@ __device__ __forceinline__ void fft_fused(const Tile &t, const FftPlan &fp, cons
         n_cur = fp.stride[j];
         tmul *= fp.radix[j];
     }
-#define X(RR) case RR: last_stage<RR, SIGN, PAD, REV, COLFAST_OUT>(t, fp, store, tid, nthr); break;
+#define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) last_stage<RR, SIGN, PAD, REV, COLFAST_OUT>(t, fp, store, tid, nthr); break;
     if (POW2) { switch (fp.radix[d - 1]) { CQT_RADIX_CASES_POW2(X) default: break; } }
     else { switch (fp.radix[d - 1]) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X

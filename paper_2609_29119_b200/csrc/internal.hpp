@@ -18,6 +18,7 @@ struct BandClass {
     int threads = 0;         // threads per CTA
     int min_blocks = 1;      // CTAs per SM the kernel instantiation is compiled for (register budget)
     int items_per_cta = 1;   // > 1: one warp per (band, signal) item
+    int max_radix = 16;      // largest butterfly radix in the class's plans
     int max_elems = 0;       // shared-memory elements (float2) per item
     int n_bands = 0;         // bands in the class
     int32_t *d_work = nullptr;  // band indices, longest first
