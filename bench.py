@@ -204,6 +204,20 @@ def path_algorithmic_bytes(plan, w, batch, second_is_adjoint=False):
     return 2 * 4 * w.valid_len * batch + 2 * 8 * plan.coeff_count * batch + 2 * 4 * plan.table_length
 
 
+def path_algorithmic_flops(plan, w, batch):
+    """Radix-2 operation count of one step (two transforms): per signal 2.5 N log2(N/2) for each packed long FFT,
+    5 M log2 M for each band transform, 16 per support entry for the window multiply and the fold / overlap-add."""
+    import math
+    bands = plan.bands()
+    per_signal = 2.0 * (2.5 * w.N * math.log2(w.N / 2.0) + sum(5.0 * b.M * math.log2(b.M) for b in bands)) \
+        + 2.0 * 16.0 * sum(b.support for b in bands)
+    return per_signal * batch
+
+
+# FP32 peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop (FMA) x 1.965 GHz
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
 def make_plan(w, device):
     from paper_2609_29119_b200 import Plan, multires_bands
     if w.sections:
@@ -401,6 +415,11 @@ def run_ours(args, w):
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
                      "frac": dom_gbs / peak, "traffic": traffic, "peak_kind": peak_kind,
                      "path_achieved": path_gbs, "path_frac": path_gbs / peak, "path_alg_bytes": path_bytes},
+        # the path is issue-bound on the CUDA cores, not bandwidth-bound: the same step against their FP32 peak
+        "roofline_alu": {"bound": "alu", "achieved": path_algorithmic_flops(plan, w, batch) / (ms / K * 1e-3) / 1e12,
+                         "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s", "peak_kind": "148 SMs x 128 lanes x 2 x 1.965 GHz",
+                         "frac": path_algorithmic_flops(plan, w, batch) / (ms / K * 1e-3) / 1e12 / FP32_PEAK_TFLOPS,
+                         "flops_per_step": path_algorithmic_flops(plan, w, batch)},
         "kernels": kernels,
         "cpu_baseline": cpu,
     }
