@@ -3,7 +3,10 @@
 
 A step is one pass of the whole hot path over one batch: cqt_analyse then cqt_synthesise of
 every signal of the workload (default: 16 stereo clips of 10 s at 44.1 kHz, N = 2^19, 24 bins
-per octave).  Prints one JSON line ("Measurement").
+per octave).  Prints one JSON line: throughput in true samples per second, the same measured end to end from
+pinned host buffers, the step replayed as a CUDA graph, per-kernel durations, the dominant kernel and the whole
+step against the measured HBM copy bandwidth and the FP32 peak, SM clocks sampled during the timed region, and
+the CPU oracle timed on a bounded sample.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload configN]
 
