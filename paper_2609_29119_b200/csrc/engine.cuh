@@ -317,13 +317,27 @@ __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, c
     const uint32_t smagic = fp.smagic[j], k1magic = fp.k1magic[j];
     const int k1div = fp.k1div[j], logC = fp.logC;
     const bool padded = PAD && fp.pad_delta != 0;
+    // Short strides: blocks of one first-stage chunk sit a multiple of 16 elements apart, so neighbouring threads on
+    // neighbouring blocks would all hit the same banks.  Then the first-stage digit k0 runs fastest over the threads
+    // instead: chunks are s_0 + 1 elements apart (the pad), which spreads a warp over all banks.
+    const bool chunk_fastest = padded && s < 16;
+    const uint32_t r0 = fp.radix[0], r0magic = fp.rmagic[0];
     for (int w = tid; w < total; w += nthr) {
         const uint32_t b = fastdiv(w, t.ncols_magic, t.ncols);
         const uint32_t col = w - b * t.ncols;
-        const uint32_t blk = fastdiv(b, smagic, s);
-        const uint32_t np = b - blk * s;
-        uint32_t pos = blk * n_cur + np;
-        if (padded) pos += fastdiv(blk, k1magic, k1div);
+        uint32_t blk, np, pad = 0;
+        if (chunk_fastest) {
+            const uint32_t x = fastdiv(b, r0magic, r0), k0 = b - x * r0;
+            const uint32_t rest = fastdiv(x, smagic, s);
+            np = x - rest * s;
+            blk = k0 * (uint32_t)k1div + rest;
+            pad = k0;
+        } else {
+            blk = fastdiv(b, smagic, s);
+            np = b - blk * s;
+            if (padded) pad = fastdiv(blk, k1magic, k1div);
+        }
+        const uint32_t pos = blk * n_cur + np + pad;
         float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
         const uint32_t step = (uint32_t)s * (uint32_t)t.pitch;
         float re[R], im[R];
