@@ -422,6 +422,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
                 p->cls[c].work.push_back(i);
                 p->cls[c].max_elems = (int)std::max<int64_t>(p->cls[c].max_elems, elems);
                 p->cls[c].n_bands++;
+                if (bf.generic) p->cls[c].has_generic = true;
             }
         }
         if (!single) {

@@ -91,7 +91,7 @@ __device__ __forceinline__ void chirp_z_transform(float2 *buf, const FftPlan &fp
     }
 }
 
-template <int THREADS, int MINB, bool WARP, int MAXR>
+template <int THREADS, int MINB, bool WARP, int MAXR, bool GEN>
 __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
     using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
@@ -126,12 +126,14 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
         return make_float2(g * xv.x, mirrored ? -(g * xv.y) : g * xv.y);
     };
     float2 *out = a.coef + (long long)ch * a.coeff_count + br.coeff_off;
-    if (fp.generic == 2) {
+    // GEN: the class holds lengths with prime factors above 5 (only the multiple-of-4 length policy makes them);
+    // the other instantiations leave the chirp-z and direct-sum code out
+    if (GEN && fp.generic == 2) {
         auto store_c = [&](int n, int, float2 v) { out[n] = v; };
         chirp_z_transform<+1, Sync>(buf, fp, a.ffts, a.tw, load, store_c, a.dbg, tid, nthr);
         return;
     }
-    if (fp.generic) {
+    if (GEN && fp.generic) {
         float2 *alt = buf + M;
         for (int m = tid; m < M; m += nthr) buf[m] = load(m, 0);
         Sync::sync();
@@ -183,7 +185,7 @@ struct RegularStore {
     }
 };
 
-template <int THREADS, int MINB, bool WARP, int MAXR>
+template <int THREADS, int MINB, bool WARP, int MAXR, bool GEN>
 __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandArgs a) {
     using G = Group<WARP>;
     using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
@@ -223,11 +225,13 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
         const float h = __ldg(tab + (d - br.d0));
         if (CQT_CHK(a.dbg, 306, (long long)br.y_off + k, a.y_pitch)) Y[k] = make_float2(h * u.x, h * u.y);
     };
-    if (fp.generic == 2) {
+    // GEN: the class holds lengths with prime factors above 5 (only the multiple-of-4 length policy makes them);
+    // the other instantiations leave the chirp-z and direct-sum code out
+    if (GEN && fp.generic == 2) {
         chirp_z_transform<-1, Sync>(buf, fp, a.ffts, a.tw, load, store, a.dbg, tid, nthr);
         return;
     }
-    if (fp.generic) {
+    if (GEN && fp.generic) {
         float2 *alt = buf + M;
         for (int n = tid; n < M; n += nthr) buf[n] = load(n, 0);
         Sync::sync();
@@ -276,9 +280,14 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
 
 template <bool ANALYSIS>
 static const void *class_kernel(const BandClass &c) {
-#define X(T, B, W, R)                                                                        \
-    if (c.threads == T && c.min_blocks == B && (c.items_per_cta > 1) == W && c.max_radix <= R) \
-        return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W, R> : (const void *)bands_to_spectrum_kernel<T, B, W, R>;
+#define X(T, B, W, R)                                                                          \
+    if (c.threads == T && c.min_blocks == B && (c.items_per_cta > 1) == W && c.max_radix <= R) { \
+        if (c.has_generic)                                                                     \
+            return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W, R, true>       \
+                            : (const void *)bands_to_spectrum_kernel<T, B, W, R, true>;        \
+        return ANALYSIS ? (const void *)bands_from_spectrum_kernel<T, B, W, R, false>          \
+                        : (const void *)bands_to_spectrum_kernel<T, B, W, R, false>;           \
+    }
     CQT_KERNEL_TABLE(X)
 #undef X
     return nullptr;

@@ -19,6 +19,7 @@ struct BandClass {
     int min_blocks = 1;      // CTAs per SM the kernel instantiation is compiled for (register budget)
     int items_per_cta = 1;   // > 1: one warp per (band, signal) item
     int max_radix = 16;      // largest butterfly radix in the class's plans
+    bool has_generic = false; // some band of the class has a prime factor above 5 (direct-sum stage or chirp-z)
     int max_elems = 0;       // shared-memory elements (float2) per item
     int n_bands = 0;         // bands in the class
     int32_t *d_work = nullptr;  // band indices, longest first
