@@ -10,8 +10,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libcqt_b200.so")
-SOURCES = ["layout.cpp", "api.cu", "band.cu", "band_two_pass.cu", "long_fft.cu", "slicq.cu", "static_ws.cu"]
-HEADERS = ["layout.hpp", "plan_types.h", "internal.hpp", "engine.cuh", "codelets_gen.cuh",
+SOURCES = ["layout.cpp", "api.cu", "band.cu", "band_analysis.cu", "band_synthesis.cu", "band_two_pass.cu", "long_fft.cu",
+           "slicq.cu", "static_ws.cu"]
+HEADERS = ["layout.hpp", "plan_types.h", "internal.hpp", "engine.cuh", "band_common.cuh", "static_fft.cuh", "codelets_gen.cuh",
            os.path.join("..", "..", "include", "cqt.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
