@@ -89,7 +89,7 @@ __device__ __forceinline__ void stage_table(float2 *dst, const float2 *__restric
 }
 
 // Every pass exists once as a template over a compile-time Shape (radices, columns, pitch) and is instantiated
-// for the common shapes plus the run-time planned fallback; the kernels pick the instantiation that matches.
+// for the common shapes plus the run-time planned fallback.
 using DynShape = Shape<0, 0, 0, 0, 0>;
 using Sh_16_16_8_8_9 = Shape<16, 16, 8, 8, 9>;
 using Sh_8_8_8_16_16 = Shape<8, 8, 8, 16, 16>;
@@ -106,14 +106,7 @@ using Sh_16_16_1_16_17 = Shape<16, 16, 1, 16, 17>;
 using Sh_16_8_1_16_17 = Shape<16, 8, 1, 16, 17>;
 using Sh_16_8_8_8_9 = Shape<16, 8, 8, 8, 9>;
 
-#define CQT_DISPATCH_SHAPES(BODY, FP, NC, ...)                                   \
-    do {                                                                         \
-        if (false) {}                                                            \
-        CQT_SHAPE_LIST(BODY, FP, NC, __VA_ARGS__)                                \
-        else BODY<DynShape>(__VA_ARGS__);                                        \
-    } while (0)
-#define CQT_TRY_SHAPE(BODY, FP, NC, SH, ...) else if (SH::matches(FP, NC)) BODY<SH>(__VA_ARGS__);
-
+// The host picks the instantiation that matches the plan (pick_kernel below): a kernel holds the code of one shape only.
 // ---------------------------------------------------------------- forward, pass C
 template <class SH>
 __device__ __forceinline__ void cols_fwd_body(const LongArgs &a, const FftPlan &fp, float2 *buf, const float2 *tws,
@@ -134,6 +127,7 @@ __device__ __forceinline__ void cols_fwd_body(const LongArgs &a, const FftPlan &
     }
 }
 
+template <class SH>
 __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
@@ -145,13 +139,7 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     float2 *wl = tws + fp.M;
     stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
-#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_16, __VA_ARGS__)          \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_16, __VA_ARGS__)        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_16, __VA_ARGS__)         \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_8, __VA_ARGS__)           \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_8_8_8, __VA_ARGS__)
-    CQT_DISPATCH_SHAPES(cols_fwd_body, fp, TW, a, fp, buf, tws, wl, j2_0, ch, tid, nthr);
+    cols_fwd_body<SH>(a, fp, buf, tws, wl, j2_0, ch, tid, nthr);
 }
 
 // rows owned by CTA t of the forward row kernel: first set TWr*t + i, second set A - TWr*t - TWr + i
@@ -225,6 +213,7 @@ __device__ __forceinline__ void rows_fwd_body(const LongArgs &a, const FftPlan &
     }
 }
 
+template <class SH>
 __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
@@ -237,13 +226,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     float2 *wn = tws + fp.M;
     stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
-#undef CQT_SHAPE_LIST
-#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_18_19, __VA_ARGS__)          \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_18_19, __VA_ARGS__)        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_18_19, __VA_ARGS__)         \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_10_11, __VA_ARGS__)
-    CQT_DISPATCH_SHAPES(rows_fwd_body, fp, ncols, a, fp, buf, tws, wn, t, ch, tid, nthr);
+    rows_fwd_body<SH>(a, fp, buf, tws, wn, t, ch, tid, nthr);
 }
 
 // ---------------------------------------------------------------- inverse: overlap-add + retangle
@@ -357,6 +340,7 @@ __device__ __forceinline__ void rows_inv_body(const LongArgs &a, const FftPlan &
     }
 }
 
+template <class SH>
 __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
@@ -369,13 +353,7 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     float2 *wl = tws + fp.M;
     stage_full(tws, a.tw, fp, tid, nthr);
     if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
-#undef CQT_SHAPE_LIST
-#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_17, __VA_ARGS__)          \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_17, __VA_ARGS__)        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_17, __VA_ARGS__)         \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_9, __VA_ARGS__)
-    CQT_DISPATCH_SHAPES(rows_inv_body, fp, ncols, a, fp, buf, tws, wl, t, ch, tid, nthr);
+    rows_inv_body<SH>(a, fp, buf, tws, wl, t, ch, tid, nthr);
 }
 
 // ---------------------------------------------------------------- inverse, pass C' (+ unpack)
@@ -399,6 +377,7 @@ __device__ __forceinline__ void cols_inv_body(const LongArgs &a, const FftPlan &
     }
 }
 
+template <class SH>
 __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
@@ -408,16 +387,8 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)a.A * (TW | 1);
     stage_full(tws, a.tw, fp, tid, nthr);
-#undef CQT_SHAPE_LIST
-#define CQT_SHAPE_LIST(BODY, FP, NC, ...)                                        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_8_8_8_16_17, __VA_ARGS__)          \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_1_16_17, __VA_ARGS__)        \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_1_16_17, __VA_ARGS__)         \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_8_8_8_9, __VA_ARGS__)           \
-    CQT_TRY_SHAPE(BODY, FP, NC, Sh_16_16_8_8_9, __VA_ARGS__)
-    CQT_DISPATCH_SHAPES(cols_inv_body, fp, TW, a, fp, buf, tws, j2_0, ch, tid, nthr);
+    cols_inv_body<SH>(a, fp, buf, tws, j2_0, ch, tid, nthr);
 }
-#undef CQT_SHAPE_LIST
 
 // ---------------------------------------------------------------- host side
 static uint32_t magic_of(uint32_t d) { return d <= 1 ? 0u : (uint32_t)(((1ull << 32) + d - 1) / d); }
@@ -474,6 +445,46 @@ static size_t cols_smem(const cqt_plan &p) {
     return ((size_t)lf.A * (lf.tw_cols | 1) + plan_tw(p, lf.fft_A) + lf.n_lp) * 8;   // odd pitch in the inverse pass
 }
 
+
+// first shape of the list that matches the plan, else the run-time planned instantiation
+template <template <class> class K, class... SHs>
+struct PickKernel;
+template <template <class> class K>
+struct PickKernel<K> {
+    static const void *get(const FftPlan &, int) { return (const void *)K<DynShape>::fn; }
+};
+template <template <class> class K, class SH, class... Rest>
+struct PickKernel<K, SH, Rest...> {
+    static const void *get(const FftPlan &fp, int ncols) {
+        return SH::matches(fp, ncols) ? (const void *)K<SH>::fn : PickKernel<K, Rest...>::get(fp, ncols);
+    }
+};
+template <class SH> struct ColsFwdK { static constexpr auto fn = rfft_cols_fwd_kernel<SH>; };
+template <class SH> struct RowsFwdK { static constexpr auto fn = rfft_rows_fwd_kernel<SH>; };
+template <class SH> struct RowsInvK { static constexpr auto fn = irfft_rows_kernel<SH>; };
+template <class SH> struct ColsInvK { static constexpr auto fn = irfft_cols_kernel<SH>; };
+
+static const void *cols_fwd_fn(const cqt_plan &p) {
+    return PickKernel<ColsFwdK, Sh_8_8_8_16_16, Sh_16_16_1_16_16, Sh_16_8_1_16_16, Sh_16_8_8_8_8, Sh_16_16_8_8_8>::get(
+        p.ffts[p.lf.fft_A], p.lf.tw_cols);
+}
+static const void *rows_fwd_fn(const cqt_plan &p) {
+    const int ncols = p.lf.A == 1 ? 1 : 2 * p.lf.tw_rows + 2;
+    return PickKernel<RowsFwdK, Sh_8_8_8_18_19, Sh_16_16_1_18_19, Sh_16_8_1_18_19, Sh_16_8_8_10_11>::get(p.ffts[p.lf.fft_B], ncols);
+}
+static const void *rows_inv_fn(const cqt_plan &p) {
+    const int ncols = p.lf.A == 1 ? 1 : p.lf.tw_rows_inv;
+    return PickKernel<RowsInvK, Sh_8_8_8_16_17, Sh_16_16_1_16_17, Sh_16_8_1_16_17, Sh_16_8_8_8_9>::get(p.ffts[p.lf.fft_B], ncols);
+}
+static const void *cols_inv_fn(const cqt_plan &p) {
+    return PickKernel<ColsInvK, Sh_8_8_8_16_17, Sh_16_16_1_16_17, Sh_16_8_1_16_17, Sh_16_8_8_8_9, Sh_16_16_8_8_9>::get(
+        p.ffts[p.lf.fft_A], p.lf.tw_cols);
+}
+static cudaError_t launch_long(const void *fn, dim3 grid, int threads, size_t smem, LongArgs &a, cudaStream_t st) {
+    void *args[] = {&a};
+    return cudaLaunchKernel(fn, grid, dim3((unsigned)threads), args, smem, st);
+}
+
 static int threads_for(size_t butterflies) {
     int t = 64;
     while (t < 512 && (size_t)t < butterflies) t *= 2;
@@ -489,17 +500,17 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
     const LongFft &lf = p.lf;
     if (lf.A > 1) {
         dim3 grid((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
-        rfft_cols_fwd_kernel<<<grid, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), st>>>(a);
+        launch_long(cols_fwd_fn(p), grid, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), a, st);
         note_launch(p, "rfft_cols_fwd", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         a.rows_magic = magic_of(2 * lf.tw_rows + 2);
         dim3 grid2((unsigned)(lf.A / (2 * lf.tw_rows)), (unsigned)batch);
-        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows + 2) / 8), rows_fwd_smem(p), st>>>(a);
+        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows + 2) / 8), rows_fwd_smem(p), a, st);
     } else {
         a.rows_magic = 0;
         dim3 grid2(1, (unsigned)batch);
-        rfft_rows_fwd_kernel<<<grid2, threads_for((size_t)lf.B / 8), rows_fwd_smem(p), st>>>(a);
+        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B / 8), rows_fwd_smem(p), a, st);
     }
     note_launch(p, "rfft_rows_fwd", st);
     return cudaGetLastError();
@@ -525,17 +536,17 @@ cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, f
         a.rows_magic = magic_of(lf.tw_rows_inv);
         a.tw_rows = lf.tw_rows_inv;
         dim3 grid((unsigned)(lf.A / lf.tw_rows_inv), (unsigned)batch);
-        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B * lf.tw_rows_inv / 8), rows_inv_smem(p), st>>>(a);
+        launch_long(rows_inv_fn(p), grid, threads_for((size_t)lf.B * lf.tw_rows_inv / 8), rows_inv_smem(p), a, st);
         note_launch(p, "irfft_rows", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         dim3 grid2((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
-        irfft_cols_kernel<<<grid2, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), st>>>(a);
+        launch_long(cols_inv_fn(p), grid2, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), a, st);
         note_launch(p, "irfft_cols", st);
     } else {
         a.rows_magic = 0;
         dim3 grid(1, (unsigned)batch);
-        irfft_rows_kernel<<<grid, threads_for((size_t)lf.B / 8), rows_inv_smem(p), st>>>(a);
+        launch_long(rows_inv_fn(p), grid, threads_for((size_t)lf.B / 8), rows_inv_smem(p), a, st);
         note_launch(p, "irfft_rows", st);
     }
     return cudaGetLastError();
@@ -543,14 +554,14 @@ cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, f
 
 cudaError_t configure_long_fft_kernels(const cqt_plan &p) {
     cudaError_t e;
-    e = cudaFuncSetAttribute(rfft_rows_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_fwd_smem(p));
+    e = cudaFuncSetAttribute(rows_fwd_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_fwd_smem(p));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(irfft_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_inv_smem(p));
+    e = cudaFuncSetAttribute(rows_inv_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_inv_smem(p));
     if (e != cudaSuccess) return e;
     if (p.lf.A > 1) {
-        e = cudaFuncSetAttribute(rfft_cols_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
+        e = cudaFuncSetAttribute(cols_fwd_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(irfft_cols_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
+        e = cudaFuncSetAttribute(cols_inv_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
     }
     return e;
 }

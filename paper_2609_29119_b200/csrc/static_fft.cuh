@@ -144,7 +144,7 @@ template <int R0_, int R1_, int R2_, int NC_, int PITCH_>
 struct Shape {
     static constexpr int R0 = R0_, R1 = R1_, R2 = R2_, NC = NC_, PITCH = PITCH_;
     static constexpr bool is_static = R0_ > 0;
-    static __device__ __forceinline__ bool matches(const FftPlan &fp, int ncols) {
+    static __host__ __device__ __forceinline__ bool matches(const FftPlan &fp, int ncols) {
         if constexpr (R0_ == 0) return true;
         else if constexpr (R2_ == 1) return ncols == NC_ && fp.nstages == 2 && fp.radix[0] == R0_ && fp.radix[1] == R1_;
         else return ncols == NC_ && fp.nstages == 3 && fp.radix[0] == R0_ && fp.radix[1] == R1_ && fp.radix[2] == R2_;
