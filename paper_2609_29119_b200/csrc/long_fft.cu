@@ -97,10 +97,6 @@ using Sh_16_16_1_16_16 = Shape<16, 16, 1, 16, 16>;
 using Sh_16_8_1_16_16 = Shape<16, 8, 1, 16, 16>;
 using Sh_16_8_8_8_8 = Shape<16, 8, 8, 8, 8>;
 using Sh_16_16_8_8_8 = Shape<16, 16, 8, 8, 8>;
-using Sh_8_8_8_18_19 = Shape<8, 8, 8, 18, 19>;
-using Sh_16_16_1_18_19 = Shape<16, 16, 1, 18, 19>;
-using Sh_16_8_1_18_19 = Shape<16, 8, 1, 18, 19>;
-using Sh_16_8_8_10_11 = Shape<16, 8, 8, 10, 11>;
 using Sh_8_8_8_16_17 = Shape<8, 8, 8, 16, 17>;
 using Sh_16_16_1_16_17 = Shape<16, 16, 1, 16, 17>;
 using Sh_16_8_1_16_17 = Shape<16, 8, 1, 16, 17>;
@@ -142,12 +138,13 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     cols_fwd_body<SH>(a, fp, buf, tws, wl, j2_0, ch, tid, nthr);
 }
 
-// rows owned by CTA t of the forward row kernel: first set TWr*t + i, second set A - TWr*t - TWr + i
-// (i < TWr owned; i == TWr is the extra, read-only row of each set; row A means row 0)
+// Rows of CTA t of the forward row kernel, column r of its tile: r < TW is row TW t + 1 + r, r >= TW its mirror
+// A - (TW t + 1 + (r - TW)).  Eq. untangle pairs row k1 with row A - k1, so both operands of every output are in
+// the tile.  The last tile's row A/2 is its own mirror; the column that would repeat it holds row 0, which pairs
+// with itself too: every row sits in exactly one tile and nothing is transformed twice.
 __device__ __forceinline__ int row_of(int t, int r, int TW, int A) {
-    const int i = r <= TW ? r : r - (TW + 1);
-    const int k1 = r <= TW ? TW * t + i : A - TW * t - TW + i;
-    return k1 >= A ? k1 - A : k1;
+    const int k1 = r < TW ? TW * t + 1 + r : A - (TW * t + 1 + (r - TW));
+    return (r >= TW && 2 * k1 == A) ? 0 : k1;
 }
 
 // ---------------------------------------------------------------- forward, pass R (+ untangle)
@@ -156,7 +153,7 @@ __device__ __forceinline__ void rows_fwd_body(const LongArgs &a, const FftPlan &
                                               const float2 *wn, int t, int ch, int tid, int nthr) {
     const int A = a.A, B = a.B, TW = a.tw_rows;
     const bool direct = (A == 1);
-    const int ncols = direct ? 1 : 2 * TW + 2;
+    const int ncols = direct ? 1 : 2 * TW;
     const int pitch = SH::is_static ? SH::PITCH : (direct ? 1 : ncols + 1);   // odd: conflict-free transposing accesses
     if (direct) {
         const float *row = a.x_in + (long long)ch * a.x_stride;
@@ -178,23 +175,19 @@ __device__ __forceinline__ void rows_fwd_body(const LongArgs &a, const FftPlan &
         }
     }
     float2 *X = a.X + (long long)ch * a.x_pitch;
-    // epilogue: each thread keeps one owned row (column o) and walks k2; for rows other than k1 = 0 the partner
-    // Z_{Lp-k} sits in the mirror row at k2' = B-1-k2, whose position is the digit-wise complement B-1-pos(k2)
+    // epilogue: each thread keeps one row (column r) and walks k2; for rows other than k1 = 0 the partner
+    // Z_{Lp-k} sits in the mirror row's column at k2' = B-1-k2, whose position is the digit-wise complement B-1-pos(k2);
+    // row 0 pairs with itself at k2' = (B - k2) mod B, row A/2 with itself at B-1-k2
     const int nown = direct ? 1 : 2 * TW;
-    const int o = direct ? 0 : (tid & (nown - 1));
+    const int r = direct ? 0 : (tid & (nown - 1));
     const int kstart = direct ? tid : (tid >> a.log_own), kstep = direct ? nthr : (nthr >> a.log_own);
-    int r = 0, rp = 0;
-    if (!direct) {
-        r = o < TW ? o : o + 1;                          // skip the extra row of the first set
-        const int i = o < TW ? o : o - TW;
-        rp = o < TW ? (TW + 1) + (TW - i) : (TW - i);    // mirror row's column
-    }
     const int k1 = direct ? 0 : row_of(t, r, TW, A);
+    const int rp = (direct || k1 == 0 || 2 * k1 == A) ? r : (r < TW ? r + TW : r - TW);
     for (int k2 = kstart; k2 < B; k2 += kstep) {
         const uint32_t pos = SH::pos(fp, (uint32_t)k2);
         uint32_t posp;
-        int rpp = rp;
-        if (k1 == 0) { rpp = r; posp = k2 == 0 ? 0u : SH::pos(fp, (uint32_t)(B - k2)); }
+        const int rpp = rp;
+        if (k1 == 0) posp = k2 == 0 ? 0u : SH::pos(fp, (uint32_t)(B - k2));
         else posp = (uint32_t)(B - 1) - pos;
         const int k = k1 + A * k2;
         if (!CQT_CHK(a.dbg, 203, k, a.Lp) || !CQT_CHK(a.dbg, 204, (size_t)posp * pitch + rpp, B * pitch) ||
@@ -218,7 +211,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
     const bool direct = (a.A == 1);
-    const int ncols = direct ? 1 : 2 * a.tw_rows + 2;
+    const int ncols = direct ? 1 : 2 * a.tw_rows;
     const int pitch = direct ? 1 : ncols + 1;
     const FftPlan &fp = a.ffts[a.fft_B];
     float2 *buf = smem_long;
@@ -432,7 +425,7 @@ static size_t plan_tw(const cqt_plan &p, int fft) { return (size_t)p.ffts[fft].M
 
 static size_t rows_fwd_smem(const cqt_plan &p) {
     const LongFft &lf = p.lf;
-    const size_t data = lf.A == 1 ? (size_t)lf.B : (size_t)lf.B * (2 * lf.tw_rows + 3);
+    const size_t data = lf.A == 1 ? (size_t)lf.B : (size_t)lf.B * (2 * lf.tw_rows + 1);
     return (data + plan_tw(p, lf.fft_B) + lf.n_n) * 8;
 }
 static size_t rows_inv_smem(const cqt_plan &p) {
@@ -469,8 +462,8 @@ static const void *cols_fwd_fn(const cqt_plan &p) {
         p.ffts[p.lf.fft_A], p.lf.tw_cols);
 }
 static const void *rows_fwd_fn(const cqt_plan &p) {
-    const int ncols = p.lf.A == 1 ? 1 : 2 * p.lf.tw_rows + 2;
-    return PickKernel<RowsFwdK, Sh_8_8_8_18_19, Sh_16_16_1_18_19, Sh_16_8_1_18_19, Sh_16_8_8_10_11>::get(p.ffts[p.lf.fft_B], ncols);
+    const int ncols = p.lf.A == 1 ? 1 : 2 * p.lf.tw_rows;
+    return PickKernel<RowsFwdK, Sh_8_8_8_16_17, Sh_16_16_1_16_17, Sh_16_8_1_16_17, Sh_16_8_8_8_9>::get(p.ffts[p.lf.fft_B], ncols);
 }
 static const void *rows_inv_fn(const cqt_plan &p) {
     const int ncols = p.lf.A == 1 ? 1 : p.lf.tw_rows_inv;
@@ -504,9 +497,9 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
         note_launch(p, "rfft_cols_fwd", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
-        a.rows_magic = magic_of(2 * lf.tw_rows + 2);
+        a.rows_magic = magic_of(2 * lf.tw_rows);
         dim3 grid2((unsigned)(lf.A / (2 * lf.tw_rows)), (unsigned)batch);
-        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows + 2) / 8), rows_fwd_smem(p), a, st);
+        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows) / 8), rows_fwd_smem(p), a, st);
     } else {
         a.rows_magic = 0;
         dim3 grid2(1, (unsigned)batch);
