@@ -1,19 +1,20 @@
 // Packed real FFT of length N through a complex FFT of length Lp = N/2 = A * B (Eq. pack), with
-// the conjugate-symmetric fold (Eq. untangle) in the epilogue of the last forward pass and the
-// inverse fold (Eq. retangle) plus the deterministic per-bin sum over bands in the prologue of the
-// first inverse pass.
+// the conjugate-symmetric fold (Eq. untangle) in the epilogue of the last forward pass; on the way back a
+// gather kernel sums, per bin and in fixed band order, the weighted bins of the bands covering it and applies
+// the inverse fold (Eq. retangle), then two inverse passes follow.
 //
 // Index split:  sample index j = j1 * B + j2,  bin index k = k1 + A * k2  (j1,k1 < A; j2,k2 < B).
 //   forward  pass C ("columns"): for TWc adjacent j2, A-point DFT over j1, times W_Lp^{j2 k1},
 //                                written to T[k1][j2].  First stage on registers straight from the
 //                                signal (packing on load), last stage straight to T.
 //            pass R ("rows"):    for a set of rows k1, B-point DFT over j2 gives Z[k1 + A k2];
-//                                a CTA owns TWr rows and their mirror images A - k1 (plus one
-//                                extra row each side) so both operands of Eq. untangle are in its
-//                                shared memory; writes the half spectrum X[0 .. Lp].
-//   inverse  pass R':            gathers X^_q = sum over covering bands (fixed order), forms Z_q by
-//                                Eq. retangle, inverse B-point DFT over q2, times conj W_Lp^{j2 q1},
-//                                written to T[q1][j2].
+//                                a CTA owns TWr rows and their mirror images A - k1 so both operands
+//                                of Eq. untangle are in its shared memory (see row_of); writes the half
+//                                spectrum X[0 .. Lp].
+//   inverse  gather:             one thread per bin pair (q, Lp - q): X^_q = sum over covering bands, Z_q and
+//                                Z_{Lp-q} by Eq. retangle.
+//            pass R':            inverse B-point DFT over q2, times conj W_Lp^{j2 q1}, written transposed to
+//                                Tinv[j2][q1].
 //            pass C':            inverse A-point DFT over q1, scaled, unpacked to x[2j], x[2j+1].
 // When Lp is small (A == 1) the row kernels read / write the signal directly and passes C, C' vanish.
 //
