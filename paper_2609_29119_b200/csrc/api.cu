@@ -89,20 +89,20 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp, b
     fp.nstages = (int32_t)radices.size();
     int64_t n_cur = M;
     for (int j = 0; j < fp.nstages; ++j) {
-        fp.radix[j] = radices[j];
-        fp.stride[j] = (int32_t)(n_cur / radices[j]);
-        fp.rmagic[j] = magic_of((uint32_t)radices[j]);
-        fp.smagic[j] = magic_of((uint32_t)fp.stride[j]);
-        const int64_t kd = j == 0 ? 1 : fp.stride[0] / n_cur;
-        fp.k1div[j] = (int32_t)kd;
-        fp.k1magic[j] = magic_of((uint32_t)kd);
+        fp.st[j].radix = radices[j];
+        fp.st[j].stride = (int32_t)(n_cur / radices[j]);
+        fp.st[j].rmagic = magic_of((uint32_t)radices[j]);
+        fp.st[j].smagic = magic_of((uint32_t)fp.st[j].stride);
+        const int64_t kd = j == 0 ? 1 : fp.st[0].stride / n_cur;
+        fp.st[j].k1div = (int32_t)kd;
+        fp.st[j].k1magic = magic_of((uint32_t)kd);
         n_cur /= radices[j];
     }
     int logC;
     fp.tw_off = append_twiddles(tw, M, logC);
     fp.logC = logC;
     fp.tw_count = (int32_t)((1ll << logC) + (M + (1ll << logC) - 1) / (1ll << logC));
-    fp.pad_delta = (fp.nstages > 1 && (fp.stride[0] % 2 == 0)) ? 1 : 0;
+    fp.pad_delta = (fp.nstages > 1 && (fp.st[0].stride % 2 == 0)) ? 1 : 0;
     fp.tw_full_off = -1;
     if (pow2 || want_full) {
         fp.tw_full_off = (int32_t)tw.size();
@@ -112,8 +112,8 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp, b
         }
         for (int j = 0; j < fp.nstages && pow2; ++j) {
             int l = 0;
-            while ((1 << l) < fp.radix[j]) ++l;
-            fp.lg[j] = l;
+            while ((1 << l) < fp.st[j].radix) ++l;
+            fp.st[j].lg = l;
         }
     }
     return true;
@@ -142,7 +142,7 @@ void host_fft_pow2(std::vector<std::complex<double>> &v) {   // in-place radix-2
 
 int64_t host_dif_pos(const FftPlan &fp, int64_t k) {
     int64_t pos = 0, rem = k;
-    for (int j = 0; j < fp.nstages; ++j) { pos = pos * fp.radix[j] + rem % fp.radix[j]; rem /= fp.radix[j]; }
+    for (int j = 0; j < fp.nstages; ++j) { pos = pos * fp.st[j].radix + rem % fp.st[j].radix; rem /= fp.st[j].radix; }
     return pos;
 }
 
@@ -399,7 +399,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
             if (p->bands[i].fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
             // a length with a large prime factor is evaluated as a chirp-z transform (two power-of-two transforms
             // of length L >= 2M - 1 in shared memory) instead of direct sums
-            if (p->ffts[p->bands[i].fft].generic == 1 && p->ffts[p->bands[i].fft].radix[0] >= 32 && M <= 8192 &&
+            if (p->ffts[p->bands[i].fft].generic == 1 && p->ffts[p->bands[i].fft].st[0].radix >= 32 && M <= 8192 &&
                 !std::getenv("CQT_NO_CHIRP_Z")) {
                 int64_t Lz = 64;
                 while (Lz < 2 * M - 1) Lz *= 2;
@@ -413,7 +413,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
             // the length-L buffer and that plan's table for chirp-z)
             const FftPlan &bf = p->ffts[p->bands[i].fft];
             const int64_t elems = bf.generic == 2 ? bf.blu_L + p->ffts[bf.blu_fft].tw_count
-                                                  : (bf.generic ? 2 * M + bf.radix[0] : M + 16 + bf.tw_count);
+                                                  : (bf.generic ? 2 * M + bf.st[0].radix : M + 16 + bf.tw_count);
             if (elems * p->cls[c].items_per_cta > smem_cap_elems) {
                 A2 = split_two_pass(M);
                 if (!A2) { delete p; return CQT_ERR_UNSUPPORTED; }
@@ -457,7 +457,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
         for (int f : {lf.fft_A, lf.fft_B}) {
             const FftPlan &q = p->ffts[f];
             std::fprintf(stderr, "  plan %d: M %d stages %d logC %d tw_off %d tw_count %d radices", f, q.M, q.nstages, q.logC, q.tw_off, q.tw_count);
-            for (int j = 0; j < q.nstages; ++j) std::fprintf(stderr, " %d(s%d)", q.radix[j], q.stride[j]);
+            for (int j = 0; j < q.nstages; ++j) std::fprintf(stderr, " %d(s%d)", q.st[j].radix, q.st[j].stride);
             std::fprintf(stderr, "\n");
         }
         for (int c = 0; c < kNumClasses; ++c)

@@ -42,8 +42,8 @@ __device__ __forceinline__ uint32_t dif_pos(const FftPlan &fp, uint32_t k) {
     uint32_t pos = 0, rem = k;
 #pragma unroll 1
     for (int j = 0; j < fp.nstages; ++j) {
-        const uint32_t r = fp.radix[j];
-        const uint32_t q = __umulhi(rem, fp.rmagic[j]);
+        const uint32_t r = fp.st[j].radix;
+        const uint32_t q = __umulhi(rem, fp.st[j].rmagic);
         pos = pos * r + (rem - q * r);
         rem = q;
     }
@@ -140,8 +140,8 @@ __device__ void fft_dif(float2 *buf, float2 *alt, int pitch, int ncols, uint32_t
     int n_cur = M, tmul = 1;
 #pragma unroll 1
     for (int j = 0; j < fp.nstages; ++j) {
-        const int r = fp.radix[j], s = fp.stride[j];
-        const uint32_t sm = fp.smagic[j];
+        const int r = fp.st[j].radix, s = fp.st[j].stride;
+        const uint32_t sm = fp.st[j].smagic;
 #define CQT_STAGE(RR)                                                                                      \
     case RR:                                                                                               \
         dif_stage<RR, SIGN>(buf, pitch, ncols, ncols_magic, M, n_cur, s, sm, tmul, tw, logC, tid, nthr); \
@@ -232,7 +232,7 @@ __device__ __forceinline__ uint32_t dif_pos_pow2(const FftPlan &fp, uint32_t k) 
     uint32_t pos = 0, rem = k;
 #pragma unroll 1
     for (int j = 0; j < fp.nstages; ++j) {
-        const int l = fp.lg[j];
+        const int l = fp.st[j].lg;
         pos = (pos << l) | (rem & ((1u << l) - 1));
         rem >>= l;
     }
@@ -270,11 +270,12 @@ template <int R, int SIGN, bool PAD, bool COLFAST, bool DIRECT, class Sync, clas
 __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, const float2 *tw, Load load, int tid, int nthr) {
     // plan fields are read once, ahead of the loops: the plan may sit in shared memory beside the data buffer,
     // where the compiler must assume that a data store changes it
-    const int s = fp.stride[0];
+    const StageRec sr = fp.st[0];
+    const int s = sr.stride;
     const int total = s * t.ncols;
     const int spad = PAD ? s + fp.pad_delta : s;
     const int logC = fp.logC;
-    const uint32_t smagic0 = fp.smagic[0];
+    const uint32_t smagic0 = sr.smagic;
     // every thread of the group runs every round: the first round contains the barrier that makes the
     // staged twiddle table visible, placed after the operand loads so both are in flight together
     for (int base = 0; base < total; base += nthr) {
@@ -312,16 +313,17 @@ __device__ __forceinline__ void first_stage(const Tile &t, const FftPlan &fp, co
 template <int R, int SIGN, bool PAD, bool DIRECT>
 __device__ __forceinline__ void middle_stage(const Tile &t, const FftPlan &fp, const float2 *tw, int j, int n_cur, int tmul,
                                              int tid, int nthr) {
-    const int s = fp.stride[j];
+    const StageRec sr = fp.st[j];
+    const int s = sr.stride;
     const int total = (fp.M / R) * t.ncols;
-    const uint32_t smagic = fp.smagic[j], k1magic = fp.k1magic[j];
-    const int k1div = fp.k1div[j], logC = fp.logC;
+    const uint32_t smagic = sr.smagic, k1magic = sr.k1magic;
+    const int k1div = sr.k1div, logC = fp.logC;
     const bool padded = PAD && fp.pad_delta != 0;
     // Short strides: blocks of one first-stage chunk sit a multiple of 16 elements apart, so neighbouring threads on
     // neighbouring blocks would all hit the same banks.  Then the first-stage digit k0 runs fastest over the threads
     // instead: chunks are s_0 + 1 elements apart (the pad), which spreads a warp over all banks.
     const bool chunk_fastest = padded && s < 16;
-    const uint32_t r0 = fp.radix[0], r0magic = fp.rmagic[0];
+    const uint32_t r0 = fp.st[0].radix, r0magic = fp.st[0].rmagic;
     for (int w = tid; w < total; w += nthr) {
         const uint32_t b = fastdiv(w, t.ncols_magic, t.ncols);
         const uint32_t col = w - b * t.ncols;
@@ -370,8 +372,9 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
     const int total = nb * t.ncols;
     const int d = fp.nstages;
     const bool padded = PAD && fp.pad_delta != 0;
-    const uint32_t k1magic = fp.k1magic[d - 1];
-    const int k1div = fp.k1div[d - 1];
+    const StageRec sr = fp.st[d - 1];
+    const uint32_t k1magic = sr.k1magic;
+    const int k1div = sr.k1div;
     for (int w = tid; w < total; w += nthr) {
         uint32_t u, col;
         if (t.ncols == 1) { u = w; col = 0; }
@@ -385,8 +388,8 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
             b = 0;
 #pragma unroll 1
             for (int j = 0; j < d - 1; ++j) {
-                const uint32_t r = fp.radix[j];
-                const uint32_t qd = __umulhi(rem, fp.rmagic[j]);
+                const uint32_t r = fp.st[j].radix;
+                const uint32_t qd = __umulhi(rem, fp.st[j].rmagic);
                 b = b * r + (rem - qd * r);
                 rem = qd;
             }
@@ -395,8 +398,8 @@ __device__ __forceinline__ void last_stage(const Tile &t, const FftPlan &fp, Sto
             uint32_t rem = u;
 #pragma unroll 1
             for (int j = d - 2; j >= 0; --j) {
-                const uint32_t r = fp.radix[j];
-                const uint32_t qd = __umulhi(rem, fp.rmagic[j]);
+                const uint32_t r = fp.st[j].radix;
+                const uint32_t qd = __umulhi(rem, fp.st[j].rmagic);
                 klow = klow * r + (rem - qd * r);
                 rem = qd;
             }
@@ -456,12 +459,12 @@ __device__ __forceinline__ void only_stage(const Tile &t, Load load, Store store
 template <int R>
 __device__ __forceinline__ void dit_stage(const Tile &t, const FftPlan &fp, const float2 *tw, int j, int n_cur, int tmul,
                                           int tid, int nthr) {
-    const int s = fp.stride[j];
+    const int s = fp.st[j].stride;
     const int total = (fp.M / R) * t.ncols;
     for (int w = tid; w < total; w += nthr) {
         const uint32_t b = fastdiv(w, t.ncols_magic, t.ncols);
         const uint32_t col = w - b * t.ncols;
-        const uint32_t blk = fastdiv(b, fp.smagic[j], s);
+        const uint32_t blk = fastdiv(b, fp.st[j].smagic, s);
         const uint32_t np = b - blk * s;
         const uint32_t pos = blk * n_cur + np;
         float2 *p = t.buf + (pos * (uint32_t)t.pitch + col);
@@ -485,10 +488,10 @@ __device__ void fft_dit_inverse(const Tile &t, const FftPlan &fp, const float2 *
     const int d = fp.nstages;
 #pragma unroll 1
     for (int j = d - 1; j >= 0; --j) {
-        const int n_cur = j == 0 ? fp.M : fp.stride[j - 1];
+        const int n_cur = j == 0 ? fp.M : fp.st[j - 1].stride;
         int tmul = 1;
-        for (int i = 0; i < j; ++i) tmul *= fp.radix[i];
-        switch (fp.radix[j]) {
+        for (int i = 0; i < j; ++i) tmul *= fp.st[i].radix;
+        switch (fp.st[j].radix) {
             case 2: dit_stage<2>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
             case 4: dit_stage<4>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
             case 8: dit_stage<8>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
@@ -515,30 +518,30 @@ __device__ __forceinline__ void fft_fused(const Tile &t, const FftPlan &fp, cons
     if (d == 1) {
         Sync::sync();   // tables staged by the caller become visible to the functors
 #define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) only_stage<RR, SIGN>(t, load, store, tid, nthr); break;
-        if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
-        else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+        if (POW2) { switch (fp.st[0].radix) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.st[0].radix) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
         return;
     }
 #define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) first_stage<RR, SIGN, PAD, COLFAST_IN, DIRECT, Sync>(t, fp, tw, load, tid, nthr); break;
-    if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
-    else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+    if (POW2) { switch (fp.st[0].radix) { CQT_RADIX_CASES_POW2(X) default: break; } }
+    else { switch (fp.st[0].radix) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
     Sync::sync();
-    int n_cur = fp.stride[0], tmul = fp.radix[0];
+    int n_cur = fp.st[0].stride, tmul = fp.st[0].radix;
 #pragma unroll 1
     for (int j = 1; j < d - 1; ++j) {
 #define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) middle_stage<RR, SIGN, PAD, DIRECT>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
-        if (POW2) { switch (fp.radix[j]) { CQT_RADIX_CASES_POW2(X) default: break; } }
-        else { switch (fp.radix[j]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+        if (POW2) { switch (fp.st[j].radix) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.st[j].radix) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
         Sync::sync();
-        n_cur = fp.stride[j];
-        tmul *= fp.radix[j];
+        n_cur = fp.st[j].stride;
+        tmul *= fp.st[j].radix;
     }
 #define X(RR) case RR: if constexpr (POW2 || RR <= MAXR) last_stage<RR, SIGN, PAD, REV, COLFAST_OUT>(t, fp, store, tid, nthr); break;
-    if (POW2) { switch (fp.radix[d - 1]) { CQT_RADIX_CASES_POW2(X) default: break; } }
-    else { switch (fp.radix[d - 1]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+    if (POW2) { switch (fp.st[d - 1].radix) { CQT_RADIX_CASES_POW2(X) default: break; } }
+    else { switch (fp.st[d - 1].radix) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
 }
 
@@ -550,27 +553,27 @@ __device__ __forceinline__ void fft_fused_keep(const Tile &t, const FftPlan &fp,
     if (d == 1) {
         auto keep = [&](int k, int col, float2 v) { t.buf[(size_t)k * t.pitch + col] = v; };
 #define X(RR) case RR: only_stage<RR, SIGN>(t, load, keep, tid, nthr); break;
-        if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
-        else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+        if (POW2) { switch (fp.st[0].radix) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.st[0].radix) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
         Sync::sync();
         return;
     }
 #define X(RR) case RR: first_stage<RR, SIGN, false, COLFAST_IN, DIRECT, Sync>(t, fp, tw, load, tid, nthr); break;
-    if (POW2) { switch (fp.radix[0]) { CQT_RADIX_CASES_POW2(X) default: break; } }
-    else { switch (fp.radix[0]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+    if (POW2) { switch (fp.st[0].radix) { CQT_RADIX_CASES_POW2(X) default: break; } }
+    else { switch (fp.st[0].radix) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
     Sync::sync();
-    int n_cur = fp.stride[0], tmul = fp.radix[0];
+    int n_cur = fp.st[0].stride, tmul = fp.st[0].radix;
 #pragma unroll 1
     for (int j = 1; j < d; ++j) {
 #define X(RR) case RR: middle_stage<RR, SIGN, false, DIRECT>(t, fp, tw, j, n_cur, tmul, tid, nthr); break;
-        if (POW2) { switch (fp.radix[j]) { CQT_RADIX_CASES_POW2(X) default: break; } }
-        else { switch (fp.radix[j]) { CQT_RADIX_CASES_ALL(X) default: break; } }
+        if (POW2) { switch (fp.st[j].radix) { CQT_RADIX_CASES_POW2(X) default: break; } }
+        else { switch (fp.st[j].radix) { CQT_RADIX_CASES_ALL(X) default: break; } }
 #undef X
         Sync::sync();
-        n_cur = fp.stride[j];
-        tmul *= fp.radix[j];
+        n_cur = fp.st[j].stride;
+        tmul *= fp.st[j].radix;
     }
 }
 

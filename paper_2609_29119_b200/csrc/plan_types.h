@@ -12,6 +12,18 @@ constexpr int kMaxStages = 8;
 // ((k_1 r_2 + k_2) r_3 + ...) (mixed-radix digit reversal).
 // Twiddles exp(-2 pi i y / M) are the product of two table entries:
 //   tw[tw_off + (y & (C-1))] * tw[tw_off + C + (y >> logC)],  C = 1 << logC.
+// Constants of one DIF stage.  radix and rmagic come first: the digit loops of the fused last stage read just those.
+struct alignas(16) StageRec {
+    int32_t radix;      // r_j
+    uint32_t rmagic;    // ceil(2^32 / r_j)
+    int32_t stride;     // s_j
+    uint32_t smagic;    // ceil(2^32 / s_j)
+    int32_t k1div;      // s_0 / n_j: butterfly blocks of stage j per first-stage output digit
+    uint32_t k1magic;
+    int32_t lg;         // log2 r_j for power-of-two plans
+    int32_t pad_;
+};
+
 struct FftPlan {
     int32_t M;
     int32_t nstages;
@@ -21,13 +33,7 @@ struct FftPlan {
     int32_t tw_count;               // entries of the two-level table (C + ceil(M / C))
     int32_t pad_delta;              // 1 if single-column buffers skip one element per s_0 positions (bank spread)
     int32_t tw_full_off;            // power-of-two plans: offset of the full table exp(-2 pi i y / M), y < M; else -1
-    int32_t radix[kMaxStages];
-    int32_t stride[kMaxStages];     // s_j
-    uint32_t rmagic[kMaxStages];    // ceil(2^32 / r_j)
-    uint32_t smagic[kMaxStages];    // ceil(2^32 / s_j)
-    int32_t k1div[kMaxStages];      // s_0 / n_j: butterfly blocks of stage j per first-stage output digit
-    uint32_t k1magic[kMaxStages];
-    int32_t lg[kMaxStages];         // log2 r_j for power-of-two plans
+    StageRec st[kMaxStages];        // per-stage constants, one 32-byte record each (two 16-byte loads in the kernels)
     // chirp-z evaluation of a length with a large prime factor: two power-of-two transforms of length blu_L
     int32_t blu_L;                  // power of two >= 2 M - 1
     int32_t blu_fft;                // FftPlan index of the length-blu_L plan
@@ -46,7 +52,7 @@ struct BandRec {
     int32_t y_off;      // offset of the band's plane in one signal's weighted-bin scratch (entries indexed by bin)
     int32_t side;       // 0 regular, 1 DC, 2 Nyquist
     int32_t fft;        // index of the FftPlan for M (-1 for bands on the two-pass kernels)
-    int32_t pad_[2];
+    int32_t pad_[3];    // 48 bytes: the plan that follows a record in a BandItem stays 16-byte aligned
 };
 
 // A band record together with the radix plan of its length: what one work item of the band kernels needs,

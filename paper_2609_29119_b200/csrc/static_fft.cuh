@@ -146,8 +146,8 @@ struct Shape {
     static constexpr bool is_static = R0_ > 0;
     static __host__ __device__ __forceinline__ bool matches(const FftPlan &fp, int ncols) {
         if constexpr (R0_ == 0) return true;
-        else if constexpr (R2_ == 1) return ncols == NC_ && fp.nstages == 2 && fp.radix[0] == R0_ && fp.radix[1] == R1_;
-        else return ncols == NC_ && fp.nstages == 3 && fp.radix[0] == R0_ && fp.radix[1] == R1_ && fp.radix[2] == R2_;
+        else if constexpr (R2_ == 1) return ncols == NC_ && fp.nstages == 2 && fp.st[0].radix == R0_ && fp.st[1].radix == R1_;
+        else return ncols == NC_ && fp.nstages == 3 && fp.st[0].radix == R0_ && fp.st[1].radix == R1_ && fp.st[2].radix == R2_;
     }
     // position of frequency k after a KEEP transform
     static __device__ __forceinline__ uint32_t pos(const FftPlan &fp, uint32_t k) {
@@ -170,7 +170,7 @@ __device__ __forceinline__ int tile_fft3_pos(int k) {
 }
 
 __device__ __forceinline__ bool plan_is(const FftPlan &fp, int r0, int r1, int r2) {
-    return fp.nstages == 3 && fp.radix[0] == r0 && fp.radix[1] == r1 && fp.radix[2] == r2;
+    return fp.nstages == 3 && fp.st[0].radix == r0 && fp.st[1].radix == r1 && fp.st[2].radix == r2;
 }
 
 }  // namespace cqt
