@@ -121,11 +121,11 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
 cudaError_t configure_band_kernels(const cqt_plan &p) {
     for (int i = 0; i < kNumClasses; ++i) {
         const size_t s = (size_t)p.cls[i].max_elems * p.cls[i].items_per_cta * sizeof(float2);
-        if (s <= 48 * 1024) continue;
+        if (p.cls[i].n_bands == 0) continue;
         if (!class_kernel<true>(p.cls[i])) return cudaErrorInvalidDeviceFunction;
-        cudaError_t e = cudaFuncSetAttribute(class_kernel<true>(p.cls[i]), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
+        cudaError_t e = allow_dynamic_smem(class_kernel<true>(p.cls[i]), s, p);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(class_kernel<false>(p.cls[i]), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
+        e = allow_dynamic_smem(class_kernel<false>(p.cls[i]), s, p);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

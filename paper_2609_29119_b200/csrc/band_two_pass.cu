@@ -242,7 +242,7 @@ int two_pass_tile() { return kTW; }
 cudaError_t configure_two_pass_kernels(const cqt_plan &p) {
     cudaError_t e = cudaSuccess;
     auto set = [&](const void *f, size_t s) {
-        if (e == cudaSuccess && s > 48 * 1024) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s);
+        if (e == cudaSuccess) e = allow_dynamic_smem(f, s, p);
     };
     for (int g = 0; g < 2; ++g) {
         if (p.two_pass[g].bands.empty()) continue;

@@ -105,6 +105,18 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
                                 float2 *T, float2 *X, cudaStream_t st);
 cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, float2 *T, float *x, int64_t x_stride,
                                 int64_t batch, int64_t valid_len, cudaStream_t st);
+// The dynamic shared-memory limit is a property of the kernel function, shared by every plan of the process: it is
+// raised to the device maximum, not to one plan's need (a later plan needing less would otherwise lower it under an
+// earlier plan, whose launches would then fail).
+inline cudaError_t allow_dynamic_smem(const void *fn, size_t need, const cqt_plan &p) {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, fn);
+    if (e != cudaSuccess) return e;
+    const long long most = (long long)p.max_smem_optin - (long long)fa.sharedSizeBytes;   // static + dynamic share the limit
+    if ((long long)need > most) return cudaErrorInvalidValue;
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
+}
+
 cudaError_t configure_long_fft_kernels(const cqt_plan &p);
 
 // band.cu

@@ -548,14 +548,14 @@ cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, f
 
 cudaError_t configure_long_fft_kernels(const cqt_plan &p) {
     cudaError_t e;
-    e = cudaFuncSetAttribute(rows_fwd_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_fwd_smem(p));
+    e = allow_dynamic_smem(rows_fwd_fn(p), rows_fwd_smem(p), p);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(rows_inv_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_inv_smem(p));
+    e = allow_dynamic_smem(rows_inv_fn(p), rows_inv_smem(p), p);
     if (e != cudaSuccess) return e;
     if (p.lf.A > 1) {
-        e = cudaFuncSetAttribute(cols_fwd_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
+        e = allow_dynamic_smem(cols_fwd_fn(p), cols_smem(p), p);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(cols_inv_fn(p), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cols_smem(p));
+        e = allow_dynamic_smem(cols_inv_fn(p), cols_smem(p), p);
     }
     return e;
 }

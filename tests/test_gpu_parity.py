@@ -201,3 +201,27 @@ def test_plan_create_default_entry_point_and_tiny_inputs():
         assert errs.max() <= TOL
         assert snr_db(x.cpu().numpy(), y.cpu().numpy()).min() >= 120.0
     assert lib.cqt_plan_destroy(h) == 0
+
+
+def test_plans_created_later_do_not_disturb_earlier_plans():
+    """Kernel attributes (dynamic shared-memory limits) are shared by all plans of the process: a plan with small
+    needs created after one with large needs must leave the first usable; both run interleaved on two streams."""
+    wa = wl.scaled(wl.CONFIGS["config3"], channels=3)
+    wb = small_workload("later_small", N=1 << 13, valid_len=1 << 13, fs=22050.0, fmin=100.0, fmax=11025.0,
+                        bins_per_octave=12, m_policy=wl.M_SMOOTH, channels=2)
+    pa = library_plan(wa)
+    xa = _dev(wl.make_signal(wa))
+    ref_a = pa.synthesise(pa.analyse(xa, valid_len=wa.valid_len), valid_len=wa.valid_len).clone()
+    pb = library_plan(wb)                      # created after pa has run, with smaller kernels' needs
+    pc = library_plan(wl.scaled(wl.CONFIGS["table1"], channels=1))
+    xb = _dev(wl.make_signal(wb))
+    ref_b = pb.synthesise(pb.analyse(xb, valid_len=wb.valid_len), valid_len=wb.valid_len).clone()
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(5):
+        ya = pa.synthesise(pa.analyse(xa, valid_len=wa.valid_len, stream=sa), valid_len=wa.valid_len, stream=sa)
+        yb = pb.synthesise(pb.analyse(xb, valid_len=wb.valid_len, stream=sb), valid_len=wb.valid_len, stream=sb)
+        torch.cuda.synchronize()
+        assert torch.equal(ya, ref_a) and torch.equal(yb, ref_b)
+    assert snr_db(wl.make_signal(wa), ref_a.cpu().numpy()).min() >= 120.0
+    pa.close(); pb.close(); pc.close()
