@@ -24,7 +24,13 @@
  *             256-byte aligned; contents are undefined after a call.  Calls that run
  *             concurrently on different streams need different workspaces.
  *   stream    a cudaStream_t passed as void*; all transform calls are asynchronous
- *             on it and never synchronise the device.
+ *             on it and never synchronise the device.  A plan owns two helper streams
+ *             that fork from and join the caller's stream inside every call (the calls
+ *             can be captured in a CUDA graph).
+ *   threads   calls on ONE plan (or one cqt_slicq) must come from one host thread at a
+ *             time: its helper streams, events and launch counters are shared state.
+ *             Different plans may be used from different threads, and one thread may
+ *             issue calls on one plan to several streams (with distinct workspaces).
  *   errors    every function returns a cqt_status; argument errors are detected on
  *             the host before any launch; nothing throws, aborts or traps.
  *             There is no CPU fallback: without a usable CUDA device the transform
