@@ -164,3 +164,93 @@ def test_band_list_builder_matches_constant_q():
     for j, (x, y) in enumerate(zip(b.bands[1:-1], g.bands[1:-1])):
         same = [b.bands[1 + i].M for i in range(len(c)) if groups[i] == groups[j]]
         assert y.M == max(same) >= x.M
+
+
+# ---- pins for the aggregate weight a_k and the dual windows h (Sec. 2: a_k = sum_lambda M_lambda g^2, h = M g / a)
+
+def _hand_layout():
+    """Four bands on N = 16 with unequal lengths, small enough to work out by hand."""
+    N = 16
+    bands = [
+        orc.Band(kc=0, d=np.array([-1, 0, 1]), g=np.array([1.0, 1.0, 1.0]), M=4, sideband=1),
+        orc.Band(kc=2, d=np.array([-1, 0, 1]), g=np.array([0.5, 1.0, 0.5]), M=4),
+        orc.Band(kc=4, d=np.array([-2, -1, 0, 1, 2]), g=np.array([0.25, 0.5, 1.0, 0.5, 0.25]), M=8),
+        orc.Band(kc=8, d=np.array([-2, -1, 0, 1, 2]), g=np.array([0.5, 1.0, 1.0, 1.0, 0.5]), M=8, sideband=2),
+    ]
+    return orc.finish_layout(orc.Layout(N=N, fs=16.0, bands=bands))
+
+
+def test_aggregate_weight_and_duals_worked_by_hand():
+    """a_k and h of a four-band layout with lengths 4, 4, 8, 8, every value worked out on paper from
+    a_k = sum M g^2 (entries on bins 0..N/2 only) and h = M g / a_k.  Dropping or misplacing the factor M changes
+    every bin two bands of different length share (1, 2, 3, 6)."""
+    lay = _hand_layout()
+    # bin:      0    1          2               3          4    5          6                7    8
+    want_a = [4.0, 4.0 + 1.0, 4.0 + 8.0 / 16, 1.0 + 2.0, 8.0, 8.0 / 4.0, 8.0 / 16 + 8.0 / 4, 8.0, 8.0]
+    assert np.allclose(lay.a, want_a, rtol=0, atol=1e-15)
+    want_h = [
+        [0.0, 1.0, 0.8],                                   # DC band: the entry on bin -1 has no dual weight
+        [0.4, 4.0 / 4.5, 2.0 / 3.0],
+        [2.0 / 4.5, 4.0 / 3.0, 1.0, 2.0, 2.0 / 2.5],
+        [4.0 / 2.5, 1.0, 1.0, 0.0, 0.0],                    # Nyquist band: entries above N/2 have none
+    ]
+    for bd, wh in zip(lay.bands, want_h):
+        assert np.allclose(bd.h, wh, rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("kstar", [40, 57, 73, 100])
+def test_aggregate_weight_from_analysis_energy(kstar):
+    """x_j = cos(2 pi k* j / N) on an interior bin that only regular bands cover: each covering band has
+    |c_lambda[n]| = (N/2) g[k* - kc] / M for all n (cosine closed form), so ||c_lambda||^2 = (N^2/4) g^2 / M and
+    sum_lambda M^2 ||c_lambda||^2 = (N^2/4) sum_lambda M g^2 = (N^2/4) a_{k*}.  The left side comes from the
+    analysis alone (pinned by the time-domain atoms); the right side is the layout's a_k."""
+    lay = orc.build_layout(fs=256.0, fmin=6.0, fmax=128.0, bins_per_octave=6, N=256, policy=orc.M_SMOOTH)
+    N = lay.N
+    covering = [bd for bd in lay.bands if bd.kc + bd.d[0] <= kstar <= bd.kc + bd.d[-1]]
+    assert covering and all(bd.sideband == 0 for bd in covering)
+    assert len({bd.M for bd in covering}) >= 1
+    c = orc.analyse(lay, np.cos(2 * np.pi * kstar * np.arange(N) / N))
+    lhs = sum(bd.M ** 2 * np.sum(np.abs(cb) ** 2) for bd, cb in zip(lay.bands, c))
+    assert abs(lhs - (N * N / 4.0) * lay.a[kstar]) <= 1e-12 * lhs
+
+
+def test_dual_is_the_length_weighted_least_squares_inverse():
+    """With D = diag(M_lambda) on the coefficients, sum_lambda M^2 T_lambda^H T_lambda = F^H diag(a) F, so the
+    synthesis of Sec. 2 with h = M g / a is the weighted least-squares inverse (D T)^+ D of the analysis
+    matrix.  Checked column by column on the real matrices of a small layout, for the bands whose support
+    touches no sideband's support (the sidebands' entries outside bins 0..N/2 carry no dual weight, which
+    is a different, equally exact inverse there).  A dual without the factor M, h = g / sum g^2, is also an
+    exact inverse but not this one: it fails here wherever two bands of different length overlap."""
+    lay = orc.build_layout(fs=64.0, fmin=6.0, fmax=32.0, bins_per_octave=4, N=64, policy=orc.M_MULT4)
+    N, P = lay.N, lay.coeff_count
+
+    def flat(c):
+        v = np.concatenate([np.asarray(cb).ravel() for cb in c])
+        return np.concatenate([v.real, v.imag])
+
+    def unflat(v):
+        z = v[:P] + 1j * v[P:]
+        out, o = [], 0
+        for bd in lay.bands:
+            out.append(z[o:o + bd.M]); o += bd.M
+        return out
+
+    T = np.stack([flat(orc.analyse(lay, e)) for e in np.eye(N)], axis=1)            # [2P, N]
+    S = np.stack([orc.synthesise(lay, unflat(e)) for e in np.eye(2 * P)], axis=1)   # [N, 2P]
+    m = np.concatenate([np.full(bd.M, float(bd.M)) for bd in lay.bands])
+    D = np.diag(np.concatenate([m, m]))
+    W = np.linalg.pinv(D @ T) @ D
+    side_bins = set()
+    for bd in lay.bands:
+        if bd.sideband:
+            side_bins |= set(int(abs(k)) if k <= N // 2 else int(N - k) for k in bd.kc + bd.d)
+    checked, lengths, o = 0, set(), 0
+    for bd in lay.bands:
+        cols = np.r_[o:o + bd.M, P + o:P + o + bd.M]
+        o += bd.M
+        if bd.sideband or side_bins & set(int(k) for k in bd.kc + bd.d):
+            continue
+        assert np.allclose(S[:, cols], W[:, cols], rtol=0, atol=1e-13)
+        checked += 1
+        lengths.add(bd.M)
+    assert checked >= 5 and len(lengths) >= 2
