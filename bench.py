@@ -232,12 +232,15 @@ def path_algorithmic_flops(plan, w, batch):
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
 
+TUNING = {}   # fields of cqt_plan_tuning set with --tune (kernel-family comparisons)
+
+
 def make_plan(w, device):
     from paper_2609_29119_b200 import Plan, multires_bands
     if w.sections:
         cen, wid, octave = multires_bands(w.fs, w.fmin, w.N, w.sections, w.min_win)
         return Plan.from_bands(w.fs, w.N, cen, wid, octave, window=w.window, m_policy=w.m_policy, device=device)
-    return Plan(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, m_policy=w.m_policy, min_win=w.min_win,
+    return Plan(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, m_policy=w.m_policy, min_win=w.min_win, **TUNING,
                 device=device)
 
 
@@ -593,7 +596,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--single", action="store_true", help="table1: one batch size through the standard step loop instead of the sweep")
     ap.add_argument("--cpu-budget-macs", type=float, default=1.2e8)
+    ap.add_argument("--tune", action="append", default=[], metavar="FIELD=VALUE",
+                    help="a field of cqt_plan_tuning (max_cta_elems, two_pass_min); "
+                         "the defaults are what the library ships with")
     args = ap.parse_args()
+    for kv in args.tune:
+        k, v = kv.split("=")
+        TUNING[k] = int(v)
     w = wl.CONFIGS[args.workload]
     if args.channels:
         w = wl.scaled(w, channels=args.channels)

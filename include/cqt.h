@@ -130,6 +130,18 @@ typedef struct cqt_slicq cqt_slicq;
 cqt_status cqt_plan_create(double fs, double fmin, double fmax, int bins_per_octave, int64_t L,
                            cqt_window window, cqt_plan **out);
 cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out);
+/*
+ * The same with the few choices of the plan builder that are not part of the transform's definition: every
+ * setting computes the same coefficients up to fp32 rounding, only the kernels that run differ.  A zero field
+ * (or tuning == NULL) means the default.  Used by the tests to reach every kernel family on small inputs and
+ * by the benchmark to compare them.
+ */
+typedef struct {
+    int64_t max_cta_elems; /* complex elements of shared memory one CTA may use for a band (>= 64): bands needing more
+                              take the two-pass kernels, which by default only bands beyond 227 KB do */
+    int64_t two_pass_min;  /* bands with more coefficients than this take the two-pass kernels */
+} cqt_plan_tuning;
+cqt_status cqt_plan_create_tuned(const cqt_plan_desc *desc, const cqt_plan_tuning *tuning, cqt_plan **out);
 /* Errors as above. */
 cqt_status cqt_plan_create_bands(const cqt_band_list_desc *desc, cqt_plan **out);
 /*

@@ -29,6 +29,10 @@ class PlanDesc(C.Structure):
                 ("device", C.c_int)]
 
 
+class PlanTuning(C.Structure):
+    _fields_ = [("max_cta_elems", C.c_int64), ("two_pass_min", C.c_int64)]
+
+
 class BandListDesc(C.Structure):
     _fields_ = [("fs", C.c_double), ("L", C.c_int64), ("window", C.c_int), ("m_policy", C.c_int), ("device", C.c_int),
                 ("n_bands", C.c_int64), ("centre_hz", C.POINTER(C.c_double)), ("width_bins", C.POINTER(C.c_double)),
@@ -44,6 +48,7 @@ class BandInfo(C.Structure):
 EXPORTS = {
     "cqt_plan_create": (C.c_int, [C.c_double, C.c_double, C.c_double, C.c_int, C.c_int64, C.c_int, C.POINTER(C.c_void_p)]),
     "cqt_plan_create_ex": (C.c_int, [C.POINTER(PlanDesc), C.POINTER(C.c_void_p)]),
+    "cqt_plan_create_tuned": (C.c_int, [C.POINTER(PlanDesc), C.POINTER(PlanTuning), C.POINTER(C.c_void_p)]),
     "cqt_plan_create_bands": (C.c_int, [C.POINTER(BandListDesc), C.POINTER(C.c_void_p)]),
     "cqt_multires_bands": (C.c_int, [C.c_double, C.c_double, C.c_int64, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int,
                                      C.c_double, C.c_int64, C.POINTER(C.c_double), C.POINTER(C.c_double),
@@ -137,14 +142,21 @@ class Plan:
     """cqt_plan_create_ex / cqt_plan_destroy plus the four transforms on torch CUDA tensors."""
 
     def __init__(self, fs: float, fmin: float, fmax: float, bins_per_octave: int, L: int, window: int = WIN_HANN,
-                 m_policy: int = M_MULT4, min_win: float = 4.0, device: Optional[int] = None):
+                 m_policy: int = M_MULT4, min_win: float = 4.0, device: Optional[int] = None,
+                 max_cta_elems: int = 0, two_pass_min: int = 0):
+        """max_cta_elems, two_pass_min: the fields of cqt_plan_tuning (0 = default); either of them non-zero
+        creates the plan with cqt_plan_create_tuned."""
         self.lib = load_library()
         if device is None:
             import torch
             device = torch.cuda.current_device()
         desc = PlanDesc(fs, fmin, fmax, bins_per_octave, L, window, m_policy, min_win, device)
         h = C.c_void_p()
-        _check(self.lib.cqt_plan_create_ex(C.byref(desc), C.byref(h)), "cqt_plan_create_ex")
+        if max_cta_elems or two_pass_min:
+            tune = PlanTuning(max_cta_elems, two_pass_min)
+            _check(self.lib.cqt_plan_create_tuned(C.byref(desc), C.byref(tune), C.byref(h)), "cqt_plan_create_tuned")
+        else:
+            _check(self.lib.cqt_plan_create_ex(C.byref(desc), C.byref(h)), "cqt_plan_create_ex")
         self._adopt(h, device)
 
     @classmethod

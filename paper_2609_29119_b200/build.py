@@ -10,9 +10,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libcqt_b200.so")
-SOURCES = ["layout.cpp", "api.cu", "band.cu", "band_analysis.cu", "band_synthesis.cu", "band_two_pass.cu", "long_fft.cu",
-           "slicq.cu", "static_ws.cu"]
-HEADERS = ["layout.hpp", "plan_types.h", "internal.hpp", "engine.cuh", "band_common.cuh", "static_fft.cuh", "codelets_gen.cuh",
+SOURCES = ["layout.cpp", "api.cu", "band.cu", "band_analysis.cu", "band_synthesis.cu", "band_two_pass.cu", "long_fft.cu", "slicq.cu", "static_ws.cu"]
+HEADERS = ["layout.hpp", "plan_types.h", "internal.hpp", "engine.cuh", "band_common.cuh", 
+           "static_fft.cuh", "codelets_gen.cuh",
            os.path.join("..", "..", "include", "cqt.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
@@ -45,6 +45,14 @@ def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False
             open(stamp, "w").close()
         else:
             os.unlink(stamp)
+    # the register codelets are written by a script; the header is not under version control
+    gen = os.path.join(CSRC, "gen_codelets.py")
+    gen_out = os.path.join(CSRC, "codelets_gen.cuh")
+    if force or _stale(gen_out, [gen]):
+        res = subprocess.run([sys.executable, gen, gen_out], capture_output=True, text=True)
+        if res.returncode:
+            sys.stderr.write(res.stdout + res.stderr)
+            raise RuntimeError("gen_codelets.py failed")
     hdrs = [os.path.join(CSRC, h) for h in HEADERS]
     nvcc = _nvcc()
     jobs = []

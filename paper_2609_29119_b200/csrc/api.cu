@@ -40,24 +40,17 @@ int append_twiddles(std::vector<float2> &tw, int64_t n, int &logC) {
 const int kBandRadices[] = {16, 15, 12, 10, 9, 8, 6, 5, 4, 3, 2};
 const int kPow2Radices[] = {16, 8, 4, 2};
 
-// fewest stages, then smallest largest radix
-int g_radix_cap = 16;   // set around the planning of two-pass sub-transforms
-int max_band_radix() {
-    int cap = g_radix_cap;
-    if (const char *v = std::getenv("CQT_MAX_RADIX")) { const int r = std::atoi(v); if (r >= 5) cap = std::min(cap, r); }
-    return cap;
-}
-
-bool best_split(int64_t m, const int *radices, int nr, std::map<int64_t, std::vector<int>> &memo, std::vector<int> &out) {
+// fewest stages, then smallest largest radix; no radix above `cap`
+bool best_split(int64_t m, const int *radices, int nr, int cap, std::map<int64_t, std::vector<int>> &memo, std::vector<int> &out) {
     if (m == 1) { out.clear(); return true; }
     auto it = memo.find(m);
     if (it != memo.end()) { out = it->second; return !out.empty(); }
     std::vector<int> best;
     for (int i = 0; i < nr; ++i) {
         const int r = radices[i];
-        if (m % r || r > max_band_radix()) continue;
+        if (m % r || r > cap) continue;
         std::vector<int> sub;
-        if (!best_split(m / r, radices, nr, memo, sub)) continue;
+        if (!best_split(m / r, radices, nr, cap, memo, sub)) continue;
         sub.push_back(r);
         std::sort(sub.begin(), sub.end(), [](int a, int b) { return a > b; });
         if (best.empty() || sub.size() < best.size() || (sub.size() == best.size() && sub[0] < best[0])) best = sub;
@@ -68,7 +61,7 @@ bool best_split(int64_t m, const int *radices, int nr, std::map<int64_t, std::ve
 }
 
 // returns false if M cannot be planned
-bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp, bool want_full = false) {
+bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp, bool want_full = false, int radix_cap = 16) {
     std::memset(&fp, 0, sizeof(fp));
     fp.M = (int32_t)M;
     int64_t smooth = M, rest = 1;
@@ -82,7 +75,7 @@ bool make_fft_plan(int64_t M, bool pow2, std::vector<float2> &tw, FftPlan &fp, b
     }
     std::map<int64_t, std::vector<int>> memo;
     std::vector<int> radices;
-    if (!best_split(smooth, pow2 ? kPow2Radices : kBandRadices, pow2 ? 4 : 11, memo, radices)) return false;
+    if (!best_split(smooth, pow2 ? kPow2Radices : kBandRadices, pow2 ? 4 : 11, radix_cap, memo, radices)) return false;
     if (rest > 1) { radices.insert(radices.begin(), (int)rest); fp.generic = 1; }
     if (radices.empty()) radices.push_back(1);
     if ((int)radices.size() > kMaxStages) return false;
@@ -229,12 +222,19 @@ cqt_status cqt_plan_create(double fs, double fmin, double fmax, int bins_per_oct
     return cqt_plan_create_ex(&d, out);
 }
 
-static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out);
+static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan_tuning &tune, cqt_plan **out);
 
 static bool length_supported(int64_t N) { return is_pow2(N) && N >= 64 && N <= (1ll << 22); }
 
 cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
+    return cqt_plan_create_tuned(desc, nullptr, out);
+}
+
+cqt_status cqt_plan_create_tuned(const cqt_plan_desc *desc, const cqt_plan_tuning *tuning, cqt_plan **out) {
     if (!desc || !out) return CQT_ERR_INVALID_ARG;
+    cqt_plan_tuning tune{};
+    if (tuning) tune = *tuning;
+    if (tune.max_cta_elems < 0 || tune.two_pass_min < 0) return CQT_ERR_INVALID_ARG;
     const int64_t N = desc->L;
     if (N < 0) return CQT_ERR_INVALID_ARG;
     if (!length_supported(N)) return CQT_ERR_UNSUPPORTED;
@@ -245,7 +245,7 @@ cqt_status cqt_plan_create_ex(const cqt_plan_desc *desc, cqt_plan **out) {
     std::string why;
     int rc = build_layout(ld, p->lay, why);
     if (rc != 0) { delete p; return (cqt_status)rc; }
-    return finish_plan(p, N, desc->device, out);
+    return finish_plan(p, N, desc->device, tune, out);
 }
 
 cqt_status cqt_plan_create_bands(const cqt_band_list_desc *desc, cqt_plan **out) {
@@ -262,7 +262,7 @@ cqt_status cqt_plan_create_bands(const cqt_band_list_desc *desc, cqt_plan **out)
     std::string why;
     int rc = build_layout_bands(ld, specs, p->lay, why);
     if (rc != 0) { delete p; return (cqt_status)rc; }
-    return finish_plan(p, N, desc->device, out);
+    return finish_plan(p, N, desc->device, cqt_plan_tuning{}, out);
 }
 
 cqt_status cqt_multires_bands(double fs, double fmin, int64_t L, const int *octaves, const int *bins_per_octave,
@@ -282,7 +282,7 @@ cqt_status cqt_multires_bands(double fs, double fmin, int64_t L, const int *octa
     return CQT_OK;
 }
 
-static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out) {
+static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan_tuning &tune, cqt_plan **out) {
     p->N = N;
     p->device = device;
     const HostLayout &L = p->lay;
@@ -297,12 +297,13 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
     // ---- transform-length plans and twiddles
     std::vector<float2> tw;
     std::map<int64_t, int> fft_of;
-    auto plan_for = [&](int64_t M, bool pow2, bool full = false) -> int {
-        const int64_t key = pow2 ? -M : (full ? M + (1ll << 40) : M);
+    enum { kPlanBand = 0, kPlanPow2 = 1, kPlanFull = 2 };
+    auto plan_for = [&](int64_t M, int kind, int cap) -> int {
+        const int64_t key = M + ((int64_t)kind << 40) + ((int64_t)cap << 44);
         auto it = fft_of.find(key);
         if (it != fft_of.end()) return it->second;
         FftPlan fp;
-        if (!make_fft_plan(M, pow2, tw, fp, full)) return -1;
+        if (!make_fft_plan(M, kind == kPlanPow2, tw, fp, kind == kPlanFull, cap)) return fft_of[key] = -1;
         p->ffts.push_back(fp);
         return fft_of[key] = (int)p->ffts.size() - 1;
     };
@@ -315,8 +316,8 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
         lf.B = std::min<int64_t>(1024, 1ll << ((lg + 1) / 2));
         lf.A = lf.Lp / lf.B;
     }
-    lf.fft_B = plan_for(lf.B, true);
-    lf.fft_A = lf.A > 1 ? plan_for(lf.A, true) : lf.fft_B;
+    lf.fft_B = plan_for(lf.B, kPlanPow2, 16);
+    lf.fft_A = lf.A > 1 ? plan_for(lf.A, kPlanPow2, 16) : lf.fft_B;
     lf.tw_lp = append_twiddles(tw, lf.Lp, lf.log_lp_c);
     lf.n_lp = (int)tw.size() - lf.tw_lp;
     lf.tw_n = append_twiddles(tw, N, lf.log_n_c);
@@ -341,48 +342,39 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
     // ---- launch classes by band length
     // class 0: one warp per item, 8 items per CTA; the others one CTA per item, sized so that several CTAs
     // share an SM (64 registers per thread) except for the longest bands, which fill its shared memory
-    int limits[kNumClasses] = {128, 1024, 4096, 13500, 1 << 30};
-    int threads[kNumClasses] = {256, 64, 256, 512, 1024};
-    int minb[kNumClasses] = {4, 16, 4, 2, 1};
-    // tuning hooks (experiments): CQT_CLASSk="limit,threads,min_blocks", CQT_MAX_RADIX=r
-    for (int c = 0; c < kNumClasses; ++c) {
-        char name[32];
-        std::snprintf(name, sizeof(name), "CQT_CLASS%d", c);
-        if (const char *v = std::getenv(name)) std::sscanf(v, "%d,%d,%d", &limits[c], &threads[c], &minb[c]);
-        p->cls[c].threads = threads[c];
-        p->cls[c].min_blocks = minb[c];
-        p->cls[c].items_per_cta = c == 0 ? 8 : 1;
-        p->cls[c].max_radix = c <= 1 ? 8 : (c == 2 ? 12 : 16);
+    const int limits[kNumClasses] = {128, 1024, 4096, 13500, 1 << 30};
+    {
+        const int threads[kNumClasses] = {256, 64, 256, 512, 1024};
+        const int minb[kNumClasses] = {4, 16, 4, 2, 1};
+        for (int c = 0; c < kNumClasses; ++c) {
+            p->cls[c].threads = threads[c];
+            p->cls[c].min_blocks = minb[c];
+            p->cls[c].items_per_cta = c == 0 ? 8 : 1;
+            p->cls[c].max_radix = c <= 1 ? 8 : (c == 2 ? 12 : 16);
+        }
     }
     std::vector<int> order(L.bands.size());
     for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L.bands[a].M > L.bands[b].M; });
     int64_t smem_cap_elems = (227 * 1024) / 8;
     // test hook: a smaller cap sends shorter bands through the two-pass (huge band) kernels
-    if (const char *cap = std::getenv("CQT_TEST_MAX_CTA_ELEMS")) {
-        const long long v = std::atoll(cap);
-        if (v >= 64 && v < smem_cap_elems) smem_cap_elems = v;
-    }
+    if (tune.max_cta_elems >= 64 && tune.max_cta_elems < smem_cap_elems) smem_cap_elems = tune.max_cta_elems;
     // bands above this length take the two-pass kernels (small tiles, many CTAs per SM)
-    int64_t two_pass_min = 1ll << 40;   // by default only bands too long for one CTA's shared memory
-    if (const char *v = std::getenv("CQT_TWO_PASS_MIN")) two_pass_min = std::max<long long>(64, std::atoll(v));
+    const int64_t two_pass_min = tune.two_pass_min > 0 ? std::max<int64_t>(64, tune.two_pass_min) : (1ll << 40);
     // M = A * B with plannable factors: fewest stages, then the most balanced split; 0 if there is none
-    int tp_radix_cap = 16;
-    if (const char *v = std::getenv("CQT_TP_MAX_RADIX")) tp_radix_cap = std::max(5, std::atoi(v));
+    const int tp_radix_cap = 16;
     auto split_two_pass = [&](int64_t M) -> int64_t {
-        g_radix_cap = tp_radix_cap;
         int64_t bestA = 0;
         int best_cost = 1 << 30;
         for (int64_t a = 2; a * a <= M; ++a) {
             if (M % a || M / a > 1600) continue;
             FftPlan t1, t2;
             std::vector<float2> scratch_tw;
-            if (!make_fft_plan(a, false, scratch_tw, t1) || t1.generic) continue;
-            if (!make_fft_plan(M / a, false, scratch_tw, t2) || t2.generic) continue;
+            if (!make_fft_plan(a, false, scratch_tw, t1, false, tp_radix_cap) || t1.generic) continue;
+            if (!make_fft_plan(M / a, false, scratch_tw, t2, false, tp_radix_cap) || t2.generic) continue;
             const int cost = t1.nstages + t2.nstages;
             if (cost <= best_cost) { best_cost = cost; bestA = a; }
         }
-        g_radix_cap = 16;
         return bestA;
     };
     for (int i : order) {
@@ -393,17 +385,15 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
         int64_t A2 = 0;
         if (!single) { A2 = split_two_pass(M); single = A2 == 0; }
         if (single) {
-            g_radix_cap = p->cls[c].max_radix;   // short bands: fewer registers, more CTAs per SM
-            p->bands[i].fft = plan_for(M, false);
-            g_radix_cap = 16;
+            // short bands: fewer registers, more CTAs per SM
+            p->bands[i].fft = plan_for(M, kPlanBand, p->cls[c].max_radix);
             if (p->bands[i].fft < 0) { delete p; return CQT_ERR_UNSUPPORTED; }
             // a length with a large prime factor is evaluated as a chirp-z transform (two power-of-two transforms
             // of length L >= 2M - 1 in shared memory) instead of direct sums
-            if (p->ffts[p->bands[i].fft].generic == 1 && p->ffts[p->bands[i].fft].st[0].radix >= 32 && M <= 8192 &&
-                !std::getenv("CQT_NO_CHIRP_Z")) {
+            if (p->ffts[p->bands[i].fft].generic == 1 && p->ffts[p->bands[i].fft].st[0].radix >= 32 && M <= 8192) {
                 int64_t Lz = 64;
                 while (Lz < 2 * M - 1) Lz *= 2;
-                const int fl = plan_for(Lz, true);
+                const int fl = plan_for(Lz, kPlanPow2, 16);
                 FftPlan &bfz = p->ffts[p->bands[i].fft];
                 make_chirp_tables(M, p->ffts[fl], tw, bfz);
                 bfz.blu_fft = fl;
@@ -430,10 +420,8 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
             tb.band = i;
             tb.A = (int32_t)A2;
             tb.B = (int32_t)(M / A2);
-            g_radix_cap = tp_radix_cap;
-            tb.fft_A = plan_for(tb.A, false, true);
-            tb.fft_B = plan_for(tb.B, false, true);
-            g_radix_cap = 16;
+            tb.fft_A = plan_for(tb.A, kPlanFull, tp_radix_cap);
+            tb.fft_B = plan_for(tb.B, kPlanFull, tp_radix_cap);
             int lc = 0;
             tb.tw_m = append_twiddles(tw, M, lc);
             tb.log_m_c = lc;
@@ -447,27 +435,6 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, cqt_plan **out
             g.max_tiles_rows = std::max(g.max_tiles_rows, (tb.A + tw_tile - 1) / tw_tile);
             g.smem_cols = std::max(g.smem_cols, two_pass_smem_cols(tb));
             g.smem_rows = std::max(g.smem_rows, two_pass_smem_rows(tb));
-        }
-    }
-    if (std::getenv("CQT_VERBOSE_PLAN")) {
-        std::fprintf(stderr, "cqt plan: N %lld Lp %lld A %lld B %lld fftA %d fftB %d tw_rows %d tw_rows_inv %d tw_cols %d n_lp %d n_n %d "
-                     "logC %d %d planes %d y_plane %lld bands %zu ffts %zu tw %zu\n", (long long)N, (long long)lf.Lp,
-                     (long long)lf.A, (long long)lf.B, lf.fft_A, lf.fft_B, lf.tw_rows, lf.tw_rows_inv, lf.tw_cols, lf.n_lp,
-                     lf.n_n, lf.log_lp_c, lf.log_n_c, p->y_planes, (long long)p->y_plane, p->bands.size(), p->ffts.size(), tw.size());
-        for (int f : {lf.fft_A, lf.fft_B}) {
-            const FftPlan &q = p->ffts[f];
-            std::fprintf(stderr, "  plan %d: M %d stages %d logC %d tw_off %d tw_count %d radices", f, q.M, q.nstages, q.logC, q.tw_off, q.tw_count);
-            for (int j = 0; j < q.nstages; ++j) std::fprintf(stderr, " %d(s%d)", q.st[j].radix, q.st[j].stride);
-            std::fprintf(stderr, "\n");
-        }
-        for (int c = 0; c < kNumClasses; ++c)
-            std::fprintf(stderr, "  class %d: bands %d threads %d items %d max_elems %d\n", c, p->cls[c].n_bands, p->cls[c].threads,
-                         p->cls[c].items_per_cta, p->cls[c].max_elems);
-        for (int g = 0; g < 2; ++g) {
-            std::fprintf(stderr, "  two-pass group %d: %zu bands, smem %zu / %zu, tiles %d / %d:", g, p->two_pass[g].bands.size(),
-                         p->two_pass[g].smem_cols, p->two_pass[g].smem_rows, p->two_pass[g].max_tiles_cols, p->two_pass[g].max_tiles_rows);
-            for (const auto &b : p->two_pass[g].bands) std::fprintf(stderr, " %dx%d(%d+%d)", b.A, b.B, p->ffts[b.fft_A].nstages, p->ffts[b.fft_B].nstages);
-            std::fprintf(stderr, "\n");
         }
     }
     if (p->device < 0) { *out = p; return CQT_OK; }

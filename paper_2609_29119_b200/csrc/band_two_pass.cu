@@ -157,24 +157,14 @@ __global__ void __launch_bounds__(THREADS, MINB) band2p_rows_kernel(TwoPassArgs 
 }
 
 // group 0: both factors <= 256 (small tiles, 128 threads, many CTAs per SM); group 1: the rest
-static int small_group_min_blocks() {
-    if (const char *v = std::getenv("CQT_TP_MINB")) return std::atoi(v);
-    return 8;
-}
 template <bool ANALYSIS>
 static const void *cols_kernel(int g) {
     if (g == 1) return (const void *)band2p_cols_kernel<512, 2, ANALYSIS>;
-    const int mb = small_group_min_blocks();
-    if (mb == 4) return (const void *)band2p_cols_kernel<128, 4, ANALYSIS>;
-    if (mb == 6) return (const void *)band2p_cols_kernel<128, 6, ANALYSIS>;
     return (const void *)band2p_cols_kernel<128, 8, ANALYSIS>;
 }
 template <bool ANALYSIS>
 static const void *rows_kernel(int g) {
     if (g == 1) return (const void *)band2p_rows_kernel<512, 2, ANALYSIS>;
-    const int mb = small_group_min_blocks();
-    if (mb == 4) return (const void *)band2p_rows_kernel<128, 4, ANALYSIS>;
-    if (mb == 6) return (const void *)band2p_rows_kernel<128, 6, ANALYSIS>;
     return (const void *)band2p_rows_kernel<128, 8, ANALYSIS>;
 }
 
@@ -203,7 +193,6 @@ static cudaError_t run_group(const cqt_plan &p, int g, const float *table, bool 
     const long long tiles = (long long)std::min(grp.max_tiles_cols, grp.max_tiles_rows) * (long long)grp.bands.size();
     int cpc = 1;
     while (cpc < 8 && tiles * ((batch + 2 * cpc - 1) / (2 * cpc)) >= 6 * slots) cpc *= 2;
-    if (const char *v = std::getenv("CQT_TWO_PASS_CPC")) cpc = std::max(1, std::atoi(v));
     a.ch_per_cta = cpc;
     a.groups = (int)((batch + cpc - 1) / cpc);
     void *args[] = {&a};

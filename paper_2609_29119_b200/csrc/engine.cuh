@@ -201,7 +201,7 @@ __device__ __forceinline__ void apply_twiddle_powers(const float2 *tw, int logC,
             wr[q] = w.x;
             wi[q] = SIGN > 0 ? -w.y : w.y;
         } else {
-            const int hb = q >= 8 ? 8 : (q >= 4 ? 4 : 2), lo = q - hb;
+            const int hb = q >= 16 ? 16 : (q >= 8 ? 8 : (q >= 4 ? 4 : 2)), lo = q - hb;
             wr[q] = fmaf(wr[hb], wr[lo], -wi[hb] * wi[lo]);
             wi[q] = fmaf(wr[hb], wi[lo], wi[hb] * wr[lo]);
         }

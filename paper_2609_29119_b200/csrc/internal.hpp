@@ -12,7 +12,6 @@
 namespace cqt {
 
 constexpr int kNumClasses = 5;
-
 // Launch shape of one band-length class.
 struct BandClass {
     int threads = 0;         // threads per CTA

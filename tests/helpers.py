@@ -15,7 +15,7 @@ def oracle_layout(w: wl.Workload):
                             min_win=w.min_win)
 
 
-def library_plan(w: wl.Workload, device=None):
+def library_plan(w: wl.Workload, device=None, **tuning):
     from paper_2609_29119_b200 import Plan, multires_bands
     if w.sections:
         c, wd, octave = multires_bands(w.fs, w.fmin, w.N, w.sections, w.min_win)
@@ -24,7 +24,7 @@ def library_plan(w: wl.Workload, device=None):
         return Plan.from_bands(w.fs, w.N, [b[0] for b in w.bands], [b[1] for b in w.bands], None, window=w.window,
                                m_policy=w.m_policy, device=device)
     return Plan(w.fs, w.fmin, w.fmax, w.bins_per_octave, w.N, window=w.window, m_policy=w.m_policy,
-                min_win=w.min_win, device=device)
+                min_win=w.min_win, device=device, **tuning)
 
 
 def split_bands(lay, flat):
