@@ -324,7 +324,6 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
     lf.n_n = (int)tw.size() - lf.tw_n;
     // tile widths chosen so that two CTAs of the row kernels (three of the column kernels) share an SM
     lf.tw_rows = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.B <= 512 ? 8 : 4, lf.A / 2);
-    lf.tw_rows_inv = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.B <= 512 ? 16 : 8, lf.A);
     lf.tw_cols = lf.A == 1 ? 1 : (int)std::min<int64_t>(lf.A <= 512 ? 16 : 8, lf.B);
     lf.x_pitch = (lf.Lp + 1 + 7) / 8 * 8;
 
@@ -535,7 +534,7 @@ cqt_status cqt_plan_band_info(const cqt_plan *p, int64_t band, cqt_band_info *ou
 size_t cqt_plan_workspace_bytes(const cqt_plan *p, int64_t batch) {
     if (!p || batch <= 0) return 0;
     const int64_t t = p->lf.A > 1 ? p->lf.Lp : 0;
-    const int64_t per = t + std::max<int64_t>(p->lf.x_pitch, p->y_pitch + p->lf.Lp) + p->two_pass_pitch;
+    const int64_t per = t + std::max<int64_t>(p->lf.x_pitch, p->y_pitch) + p->two_pass_pitch;
     return (size_t)(256 + batch * per * (int64_t)sizeof(float2));
 }
 
@@ -611,7 +610,7 @@ namespace {
 
 struct Call {
     const cqt_plan *p;
-    float2 *T, *second, *zbuf, *huge;   // workspace regions
+    float2 *T, *second, *huge;   // workspace regions
     cudaStream_t st;
     int prev_dev;
 };
@@ -626,8 +625,7 @@ cqt_status begin_call(const cqt_plan *p, const void *sig, int64_t stride, int64_
     c.p = p;
     c.T = reinterpret_cast<float2 *>(ws);
     c.second = c.T + (p->lf.A > 1 ? batch * p->lf.Lp : 0);
-    c.zbuf = c.second + batch * p->y_pitch;   // packed spectrum of the inverse, after the weighted-bin planes
-    c.huge = c.second + batch * std::max<int64_t>(p->lf.x_pitch, p->y_pitch + p->lf.Lp);
+    c.huge = c.second + batch * std::max<int64_t>(p->lf.x_pitch, p->y_pitch);
     c.st = reinterpret_cast<cudaStream_t>(stream);
     if (cudaGetDevice(&c.prev_dev) != cudaSuccess) return CQT_ERR_CUDA;
     if (c.prev_dev != p->device && cudaSetDevice(p->device) != cudaSuccess) return CQT_ERR_CUDA;
@@ -658,7 +656,7 @@ cqt_status run_synthesis_form(const cqt_plan *p, const float *table, bool fold, 
     if (s != CQT_OK) return s;
     cudaError_t e = launch_two_pass_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, k.huge, batch, k.st);
     if (e == cudaSuccess) e = launch_bands_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, batch, k.st);
-    if (e == cudaSuccess) e = launch_rfft_inverse(*p, k.second, k.zbuf, k.T, x, x_stride, batch, valid_len, k.st);
+    if (e == cudaSuccess) e = launch_rfft_inverse(*p, k.second, k.T, x, x_stride, batch, valid_len, k.st);
     return end_call(k, e);
 }
 

@@ -31,8 +31,7 @@ struct LongFft {
     int tw_lp = 0, tw_n = 0;      // two-level tables of W_Lp and W_N inside the twiddle array
     int log_lp_c = 0, log_n_c = 0;
     int n_lp = 0, n_n = 0;        // entry counts of those tables
-    int tw_rows = 1;              // rows per mirrored half handled by one CTA of the forward row kernel
-    int tw_rows_inv = 1;          // rows per CTA of the inverse row kernel
+    int tw_rows = 1;              // rows per mirrored half handled by one CTA of the row kernels (forward and inverse)
     int tw_cols = 1;              // columns per CTA of the column kernels
     int64_t x_pitch = 0;          // elements per signal of the half-spectrum buffer (Lp + 1 rounded up)
 };
@@ -102,7 +101,7 @@ void note_launch(const cqt_plan &p, const char *name, cudaStream_t st);
 // long_fft.cu
 cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,
                                 float2 *T, float2 *X, cudaStream_t st);
-cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, float2 *T, float *x, int64_t x_stride,
+cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, float *x, int64_t x_stride,
                                 int64_t batch, int64_t valid_len, cudaStream_t st);
 // The dynamic shared-memory limit is a property of the kernel function, shared by every plan of the process: it is
 // raised to the device maximum, not to one plan's need (a later plan needing less would otherwise lower it under an

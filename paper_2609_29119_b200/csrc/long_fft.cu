@@ -1,7 +1,7 @@
 // Packed real FFT of length N through a complex FFT of length Lp = N/2 = A * B (Eq. pack), with
-// the conjugate-symmetric fold (Eq. untangle) in the epilogue of the last forward pass; on the way back a
-// gather kernel sums, per bin and in fixed band order, the weighted bins of the bands covering it and applies
-// the inverse fold (Eq. retangle), then two inverse passes follow.
+// the conjugate-symmetric fold (Eq. untangle) in the epilogue of the last forward pass; on the way back the
+// prologue of the first inverse pass sums, per bin and in fixed band order, the weighted bins of the bands
+// covering it and applies the inverse fold (Eq. retangle).
 //
 // Index split:  sample index j = j1 * B + j2,  bin index k = k1 + A * k2  (j1,k1 < A; j2,k2 < B).
 //   forward  pass C ("columns"): for TWc adjacent j2, A-point DFT over j1, times W_Lp^{j2 k1},
@@ -11,10 +11,10 @@
 //                                a CTA owns TWr rows and their mirror images A - k1 so both operands
 //                                of Eq. untangle are in its shared memory (see row_of); writes the half
 //                                spectrum X[0 .. Lp].
-//   inverse  gather:             one thread per bin pair (q, Lp - q): X^_q = sum over covering bands, Z_q and
-//                                Z_{Lp-q} by Eq. retangle.
-//            pass R':            inverse B-point DFT over q2, times conj W_Lp^{j2 q1}, written transposed to
-//                                Tinv[j2][q1].
+//   inverse  pass R':            a CTA owns the same rows as in forward pass R; per bin pair (q, Lp - q) it forms
+//                                X^_q = sum over covering bands once and Z_q, Z_{Lp-q} by Eq. retangle in shared
+//                                memory, then the inverse B-point DFT over q2, times conj W_Lp^{j2 q1}, written
+//                                transposed to Tinv[j2][q1].
 //            pass C':            inverse A-point DFT over q1, scaled, unpacked to x[2j], x[2j+1].
 // When Lp is small (A == 1) the row kernels read / write the signal directly and passes C, C' vanish.
 //
@@ -46,8 +46,7 @@ struct LongArgs {
     long long t_pitch;
     float2 *X;             // half spectrum rows (forward)
     long long x_pitch;
-    // inverse gather
-    float2 *Z;             // packed spectrum rows assembled by the gather kernel (inverse)
+    // inverse: overlap-add + retangle in the prologue of the row pass
     int log_b, log_own;    // log2 B, log2 (2 TWr)
     const float2 *Y;
     long long y_pitch;     // per signal
@@ -262,52 +261,111 @@ __device__ __forceinline__ float2 gather_finish(const float2 *__restrict__ Y, Ga
     return acc;
 }
 
-// One thread per pair (q, Lp - q), 0 <= q <= Lp/2: every bin of the half spectrum is summed once, both
-// packed bins of the pair follow from the same two values (Eq. retangle with w_{Lp-q} = -conj w_q):
+// One pair (q, m = Lp - q) of packed bins: both half-spectrum bins are summed once (bands in fixed order) and both
+// packed bins follow from the same two values (Eq. retangle with w_{Lp-q} = -conj w_q):
 //   Z_q      = s [ (X_q + conj X_m) + i conj(w) (X_q - conj X_m) ]
-//   Z_{Lp-q} = s [ (X_m + conj X_q) - i w (X_m - conj X_q) ],   m = Lp - q, w = exp(-2 pi i q / N), s = 1/(2 Lp)
-__global__ void __launch_bounds__(256, 8) gather_retangle_kernel(LongArgs a) {
-    const int ch = blockIdx.y;
-    const int Lp = a.Lp;
-    const int q = blockIdx.x * blockDim.x + threadIdx.x;
-    if (q > (Lp >> 1)) return;
-    const float2 *Y = a.Y + (long long)ch * a.y_pitch;
-    float2 *Z = a.Z + (long long)ch * a.t_pitch;
-    const int m = Lp - q;
-    if (!CQT_CHK(a.dbg, 205, m, Lp + 1)) return;
-    const int32_t cvq = __ldg(a.cover + q), cvm = __ldg(a.cover + m);
-    GatherLoads gq = gather_issue(a, Y, q, cvq), gm = gather_issue(a, Y, m, cvm);
+//   Z_{Lp-q} = s [ (X_m + conj X_q) - i w (X_m - conj X_q) ],   w = exp(-2 pi i q / N), s = 1/(2 Lp)
+// wn: two-level table of W_N (shared memory).
+__device__ __forceinline__ void retangle_finish(const LongArgs &a, const float2 *__restrict__ Y, const float2 *wn, int q,
+                                                GatherLoads &gq, GatherLoads &gm, float2 &zq, float2 &zm) {
     float2 xq = gather_finish(Y, gq);
     float2 xm = gather_finish(Y, gm);
     if (q == 0) { xq.y = 0.f; xm.y = 0.f; }   // bins 0 and N/2 are made real
-    const float2 w = twiddle(a.tw + a.tw_n, a.log_n_c, (uint32_t)q);
+    const float2 w = twiddle_s(wn, a.log_n_c, (uint32_t)q);
     {
         const float2 ev = make_float2(xq.x + xm.x, xq.y - xm.y);   // X_q + conj X_m
         const float2 od = make_float2(xq.x - xm.x, xq.y + xm.y);   // X_q - conj X_m
         const float2 rot = cmul(make_float2(w.y, w.x), od);        // i conj(w) = (w.y, w.x)
-        Z[q] = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
+        zq = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
     }
-    if (q != 0 && m != q) {
+    {
         const float2 ev = make_float2(xm.x + xq.x, xm.y - xq.y);   // X_m + conj X_q
         const float2 od = make_float2(xm.x - xq.x, xm.y + xq.y);   // X_m - conj X_q
         const float2 rot = cmul(make_float2(w.y, -w.x), od);       // -i w = (w.y, -w.x)
-        Z[m] = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
+        zm = make_float2(a.scale * (ev.x + rot.x), a.scale * (ev.y + rot.y));
     }
 }
+__device__ __forceinline__ void retangle_pair(const LongArgs &a, const float2 *__restrict__ Y, const float2 *wn, int q, int m,
+                                              float2 &zq, float2 &zm) {
+    const int32_t cvq = __ldg(a.cover + q), cvm = __ldg(a.cover + m);
+    GatherLoads gq = gather_issue(a, Y, q, cvq), gm = gather_issue(a, Y, m, cvm);
+    retangle_finish(a, Y, wn, q, gq, gm, zq, zm);
+}
 
-// ---------------------------------------------------------------- inverse, pass R'
+// ---------------------------------------------------------------- inverse, pass R' (overlap-add + retangle + B-point pass)
+// The tile holds TW rows q1 and their mirror rows A - q1 (the same rows as the forward row pass, see row_of), so
+// the two packed bins of every pair (q, Lp - q) lie in one tile: the prologue sums each half-spectrum bin once and
+// writes both packed bins to shared memory, then the B-point inverse pass runs in place.
 template <class SH>
 __device__ __forceinline__ void rows_inv_body(const LongArgs &a, const FftPlan &fp, float2 *buf, const float2 *tws,
-                                              const float2 *wl, int t, int ch, int tid, int nthr) {
-    const int A = a.A, B = a.B, TW = a.tw_rows;
+                                              const float2 *wl, const float2 *wn, int t, int ch, int tid, int nthr) {
+    const int A = a.A, B = a.B, TW = a.tw_rows, Lp = a.Lp;
     const bool direct = (A == 1);
-    const int ncols = direct ? 1 : TW;
-    const int pitch = SH::is_static ? SH::PITCH : (direct ? 1 : (TW | 1));
-    const float2 *Z = a.Z + (long long)ch * a.t_pitch;
-    auto load = [&](int q2, int r) -> float2 {
-        const int i = (direct ? 0 : t * TW + r) + A * q2;
-        return CQT_CHK(a.dbg, 210, i, a.Lp) ? __ldg(Z + i) : make_float2(0.f, 0.f);
-    };
+    const int ncols = direct ? 1 : 2 * TW;
+    const int pitch = SH::is_static ? SH::PITCH : (direct ? 1 : ncols + 1);
+    const float2 *Y = a.Y + (long long)ch * a.y_pitch;
+    __syncthreads();   // the table of W_N is staged
+    if (direct) {
+        for (int q = tid; q <= (Lp >> 1); q += nthr) {
+            const int m = Lp - q;
+            float2 zq, zm;
+            retangle_pair(a, Y, wn, q, m, zq, zm);
+            buf[q] = zq;
+            if (q != 0 && m != q) buf[m] = zm;
+        }
+    } else {
+        // Four pairs per thread and round: all cover words are fetched first, then the plane values of two pairs
+        // at a time, so that the dependent loads of one pair overlap those of the others.
+        const int log_tw = 31 - __clz(TW);
+        constexpr int kPairs = 4;
+        for (int base = 0; base < TW * B; base += kPairs * nthr) {
+            int q[kPairs], r[kPairs], q2[kPairs];
+            int32_t cq[kPairs], cm[kPairs];
+            bool ok[kPairs], self[kPairs];
+#pragma unroll
+            for (int u = 0; u < kPairs; ++u) {
+                const int idx = base + u * nthr + tid;
+                r[u] = idx & (TW - 1);
+                q2[u] = idx >> log_tw;
+                const int k1 = TW * t + 1 + r[u];
+                self[u] = 2 * k1 == A;           // row A/2 is its own mirror: the pairs (q2, B-1-q2) of one column
+                ok[u] = idx < TW * B && !(self[u] && q2[u] >= (B >> 1));
+                q[u] = ok[u] ? k1 + A * q2[u] : 1;
+                if (!CQT_CHK(a.dbg, 210, Lp - q[u], Lp) || !CQT_CHK(a.dbg, 211, q[u], Lp)) { ok[u] = false; q[u] = 1; }
+                cq[u] = __ldg(a.cover + q[u]);
+                cm[u] = __ldg(a.cover + (Lp - q[u]));
+            }
+#pragma unroll
+            for (int u = 0; u < kPairs; u += 2) {
+                GatherLoads g0q = gather_issue(a, Y, q[u], cq[u]), g0m = gather_issue(a, Y, Lp - q[u], cm[u]);
+                GatherLoads g1q = gather_issue(a, Y, q[u + 1], cq[u + 1]), g1m = gather_issue(a, Y, Lp - q[u + 1], cm[u + 1]);
+                float2 zq, zm;
+                retangle_finish(a, Y, wn, q[u], g0q, g0m, zq, zm);
+                if (ok[u]) {
+                    buf[q2[u] * pitch + r[u]] = zq;
+                    buf[(B - 1 - q2[u]) * pitch + (self[u] ? r[u] : r[u] + TW)] = zm;
+                }
+                retangle_finish(a, Y, wn, q[u + 1], g1q, g1m, zq, zm);
+                if (ok[u + 1]) {
+                    buf[q2[u + 1] * pitch + r[u + 1]] = zq;
+                    buf[(B - 1 - q2[u + 1]) * pitch + (self[u + 1] ? r[u + 1] : r[u + 1] + TW)] = zm;
+                }
+            }
+        }
+        if (2 * TW * (t + 1) == A) {
+            // the last tile's spare column holds row 0, which pairs with itself: bins A q2 and A (B - q2)
+            const int rz = 2 * TW - 1;
+            for (int q2 = tid; q2 <= (B >> 1); q2 += nthr) {
+                const int q = A * q2, m = Lp - q;
+                float2 zq, zm;
+                retangle_pair(a, Y, wn, q, m, zq, zm);
+                buf[q2 * pitch + rz] = zq;
+                if (q2 != 0 && m != q) buf[(B - q2) * pitch + rz] = zm;
+            }
+        }
+    }
+    __syncthreads();
+    auto load = [&](int q2, int r) -> float2 { return buf[q2 * pitch + r]; };
     if constexpr (SH::is_static) {
         auto nostore = [](int, int, float2) {};
         tile_fft_static<SH, +1, true, true>(buf, tws, load, nostore, tid, nthr);
@@ -320,13 +378,12 @@ __device__ __forceinline__ void rows_inv_body(const LongArgs &a, const FftPlan &
         for (int j = tid; j < B; j += nthr) store_packed(row, j, buf[SH::pos(fp, (uint32_t)j)], a.valid_len, a.aligned);
     } else {
         float2 *T = a.T + (long long)ch * a.t_pitch;
-        // The inverse keeps its intermediate transposed, Tinv[j2][q1]: consecutive threads take consecutive rows r, so
+        // The inverse keeps its intermediate transposed, Tinv[j2][q1]: consecutive threads take consecutive columns r, so
         // the shared-memory reads (odd pitch) are conflict-free and the 8-byte stores of a warp fall in runs of TW rows;
         // reading the digit-reversed positions of consecutive j2 instead would hit one bank 16 times.
-        const int log_tw = 31 - __clz(TW);
         for (int e = tid; e < ncols * B; e += nthr) {
-            const int j2 = e >> log_tw, r = e - (j2 << log_tw);
-            const int q1 = t * TW + r;
+            const int j2 = e >> a.log_own, r = e - (j2 << a.log_own);
+            const int q1 = row_of(t, r, TW, A);
             const float2 v = buf[SH::pos(fp, (uint32_t)j2) * (uint32_t)pitch + r];
             const float2 w = cconj(twiddle_s(wl, a.log_lp_c, (uint32_t)j2 * (uint32_t)q1));
             if (CQT_CHK(a.dbg, 207, j2 * A + q1, a.Lp)) T[j2 * A + q1] = cmul(v, w);
@@ -339,15 +396,17 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
     const bool direct = (a.A == 1);
-    const int ncols = direct ? 1 : a.tw_rows;
-    const int pitch = direct ? 1 : (a.tw_rows | 1);
+    const int ncols = direct ? 1 : 2 * a.tw_rows;
+    const int pitch = direct ? 1 : ncols + 1;
     const FftPlan &fp = a.ffts[a.fft_B];
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)a.B * pitch;
-    float2 *wl = tws + fp.M;
+    float2 *wn = tws + fp.M;
+    float2 *wl = wn + a.n_n;
     stage_full(tws, a.tw, fp, tid, nthr);
+    stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
     if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
-    rows_inv_body<SH>(a, fp, buf, tws, wl, t, ch, tid, nthr);
+    rows_inv_body<SH>(a, fp, buf, tws, wl, wn, t, ch, tid, nthr);
 }
 
 // ---------------------------------------------------------------- inverse, pass C' (+ unpack)
@@ -431,8 +490,8 @@ static size_t rows_fwd_smem(const cqt_plan &p) {
 }
 static size_t rows_inv_smem(const cqt_plan &p) {
     const LongFft &lf = p.lf;
-    const size_t data = lf.A == 1 ? (size_t)lf.B : (size_t)lf.B * (lf.tw_rows_inv | 1);
-    return (data + plan_tw(p, lf.fft_B) + (lf.A == 1 ? 0 : lf.n_lp)) * 8;
+    const size_t data = lf.A == 1 ? (size_t)lf.B : (size_t)lf.B * (2 * lf.tw_rows + 1);
+    return (data + plan_tw(p, lf.fft_B) + lf.n_n + (lf.A == 1 ? 0 : lf.n_lp)) * 8;
 }
 static size_t cols_smem(const cqt_plan &p) {
     const LongFft &lf = p.lf;
@@ -467,7 +526,7 @@ static const void *rows_fwd_fn(const cqt_plan &p) {
     return PickKernel<RowsFwdK, Sh_8_8_8_16_17, Sh_16_16_1_16_17, Sh_16_8_1_16_17, Sh_16_8_8_8_9>::get(p.ffts[p.lf.fft_B], ncols);
 }
 static const void *rows_inv_fn(const cqt_plan &p) {
-    const int ncols = p.lf.A == 1 ? 1 : p.lf.tw_rows_inv;
+    const int ncols = p.lf.A == 1 ? 1 : 2 * p.lf.tw_rows;
     return PickKernel<RowsInvK, Sh_8_8_8_16_17, Sh_16_16_1_16_17, Sh_16_8_1_16_17, Sh_16_8_8_8_9>::get(p.ffts[p.lf.fft_B], ncols);
 }
 static const void *cols_inv_fn(const cqt_plan &p) {
@@ -510,27 +569,18 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
     return cudaGetLastError();
 }
 
-cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *Z, float2 *T, float *x, int64_t x_stride,
+cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, float *x, int64_t x_stride,
                                 int64_t batch, int64_t valid_len, cudaStream_t st) {
     LongArgs a = base_args(p, valid_len, x_stride, x);
     a.x_out = x;
     a.T = T;
-    a.Z = Z;
     a.Y = Y;
     a.scale = (float)(0.5 / (double)p.lf.Lp);
     const LongFft &lf = p.lf;
-    {
-        dim3 grid((unsigned)((lf.Lp / 2 + 1 + 255) / 256), (unsigned)batch);
-        gather_retangle_kernel<<<grid, 256, 0, st>>>(a);
-        note_launch(p, "gather_retangle", st);
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
     if (lf.A > 1) {
-        a.rows_magic = magic_of(lf.tw_rows_inv);
-        a.tw_rows = lf.tw_rows_inv;
-        dim3 grid((unsigned)(lf.A / lf.tw_rows_inv), (unsigned)batch);
-        launch_long(rows_inv_fn(p), grid, threads_for((size_t)lf.B * lf.tw_rows_inv / 8), rows_inv_smem(p), a, st);
+        a.rows_magic = magic_of(2 * lf.tw_rows);
+        dim3 grid((unsigned)(lf.A / (2 * lf.tw_rows)), (unsigned)batch);
+        launch_long(rows_inv_fn(p), grid, threads_for((size_t)lf.B * (2 * lf.tw_rows) / 8), rows_inv_smem(p), a, st);
         note_launch(p, "irfft_rows", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
