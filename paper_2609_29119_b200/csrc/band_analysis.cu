@@ -56,7 +56,8 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     float2 *tws = buf + M + 16;
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
     const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
-    auto store = [&](int n, int, float2 v) { if (CQT_CHK(a.dbg, 303, n, M)) out[n] = v; };
+    // coefficients are written once and not read again by this call: streaming stores keep the L2 for the spectrum
+    auto store = [&](int n, int, float2 v) { if (CQT_CHK(a.dbg, 303, n, M)) __stcs(out + n, v); };
     if (br.side == 0) {
         // regular band: every support bin lies in 1..N/2-1; spectrum and table share the support index j = d - d0
         const float2 *Xs = X + (br.kc + br.d0);

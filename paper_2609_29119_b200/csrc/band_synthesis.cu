@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     const bool fold = a.fold && br.side != 0;
     auto load = [&](int n, int) -> float2 {
         if (!CQT_CHK(a.dbg, 304, n, M)) return make_float2(0.f, 0.f);
-        float2 v = __ldg(in + n);
+        float2 v = __ldcs(in + n);
         if (fold) v = make_float2(2.f * v.x, 0.f);
         return v;
     };
@@ -86,7 +86,8 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
         float2 *Ys = Y + (br.kc + br.d0);
         const int shift_neg = M + br.d0;
         const RegularStore store_regular{tab, Ys, last_pos, first_neg, br.d0, shift_neg};
-        auto load_regular = [&](int n, int) -> float2 { return __ldg(in + n); };
+        // coefficients are read once: streaming loads keep the L2 for the weighted-bin planes
+        auto load_regular = [&](int n, int) -> float2 { return __ldcs(in + n); };
         fft_fused<-1, Sync, false, true, false, true, false, false, MAXR>(t, fp, tws, load_regular, store_regular, tid, nthr);
         return;
     }

@@ -61,20 +61,20 @@ struct LongArgs {
 __device__ __forceinline__ float2 load_packed(const float *row, int j, int valid_len, int aligned) {
     const int i = 2 * j;
     if (i + 1 < valid_len) {
-        if (aligned) return __ldg(reinterpret_cast<const float2 *>(row + i));
-        return make_float2(__ldg(row + i), __ldg(row + i + 1));
+        if (aligned) return __ldcs(reinterpret_cast<const float2 *>(row + i));   // read once: streaming
+        return make_float2(__ldcs(row + i), __ldcs(row + i + 1));
     }
-    if (i < valid_len) return make_float2(__ldg(row + i), 0.f);
+    if (i < valid_len) return make_float2(__ldcs(row + i), 0.f);
     return make_float2(0.f, 0.f);
 }
 
 __device__ __forceinline__ void store_packed(float *row, int j, float2 v, int valid_len, int aligned) {
     const int i = 2 * j;
     if (i + 1 < valid_len) {
-        if (aligned) *reinterpret_cast<float2 *>(row + i) = v;
-        else { row[i] = v.x; row[i + 1] = v.y; }
+        if (aligned) __stcs(reinterpret_cast<float2 *>(row + i), v);
+        else { __stcs(row + i, v.x); __stcs(row + i + 1, v.y); }
     } else if (i < valid_len) {
-        row[i] = v.x;
+        __stcs(row + i, v.x);
     }
 }
 
