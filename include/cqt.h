@@ -63,7 +63,7 @@ typedef enum { CQT_WIN_HANN = 0, CQT_WIN_BLACKMAN_HARRIS = 1 } cqt_window;
 
 /* how the coefficient count M of a band follows from its support S (number of nonzero window bins) */
 typedef enum {
-    CQT_M_MULT4 = 0,  /* 4 * ceil(S / 4) */
+    CQT_M_MULT4 = 0,  /* 4 * ceil(S / 4); a band beyond 12,800 coefficients takes the CQT_M_SMOOTH length */
     CQT_M_SMOOTH = 1, /* smallest multiple of 4 of the form 2^a 3^b 5^c that is >= S */
     CQT_M_POW2 = 2    /* smallest power of two >= max(S, 4) */
 } cqt_m_policy;

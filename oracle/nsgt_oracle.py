@@ -51,6 +51,11 @@ M_POW2 = 2
 
 _BH = (0.35875, 0.48829, 0.14128, 0.01168)
 
+# The multiple-of-4 length policy is stated for 2^16-sample signals, whose bands stay below 6,400 coefficients.
+# A reading for longer transforms: a band beyond this many coefficients takes the next 5-smooth multiple of 4,
+# as under M_SMOOTH (any length >= the support keeps the frame painless).
+MAX_RAGGED_LENGTH = 12800
+
 
 # --------------------------------------------------------------------------
 # layout (Sec. 2: windows g, lengths M, aggregate weight a_k, duals h)
@@ -77,9 +82,9 @@ def _is_5_smooth(m: int) -> bool:
 
 def band_length(S: int, policy: int) -> int:
     """Coefficient count M of a band whose support has S bins (M >= S: painless case)."""
-    if policy == M_MULT4:
+    if policy == M_MULT4 and 4 * ((S + 3) // 4) <= MAX_RAGGED_LENGTH:
         return 4 * ((S + 3) // 4)
-    if policy == M_SMOOTH:
+    if policy in (M_MULT4, M_SMOOTH):
         m = 4 * ((S + 3) // 4)
         while not _is_5_smooth(m):
             m += 4
@@ -388,12 +393,14 @@ def synthesise(lay: Layout, c: Sequence[np.ndarray], bands: Optional[Sequence[in
 # real adjoints under <u,v> = Re(u^H v)   (Sec. 3.2)
 # --------------------------------------------------------------------------
 
-def analyse_adjoint(lay: Layout, ybar: Sequence[np.ndarray]) -> np.ndarray:
-    """T^dagger ybar = Re( F_N^H sum_lambda diag(g) E^T (1/M) F_M ybar_lambda ), all support entries."""
+def analyse_adjoint(lay: Layout, ybar: Sequence[np.ndarray], bands: Optional[Sequence[int]] = None) -> np.ndarray:
+    """T^dagger ybar = Re( F_N^H sum_lambda diag(g) E^T (1/M) F_M ybar_lambda ), all support entries.
+    With `bands`, ybar lists only those bands and the others contribute nothing."""
     N = lay.N
     lead = np.asarray(ybar[0]).shape[:-1]
     V = np.zeros(lead + (N,), dtype=np.complex128)
-    for b, yb in zip(lay.bands, ybar):
+    which = lay.bands if bands is None else [lay.bands[i] for i in bands]
+    for b, yb in zip(which, ybar):
         yb = np.asarray(yb, dtype=np.complex128)
         U = _direct_band_sum(yb, np.arange(b.M, dtype=np.int64), b.d % b.M, b.M, -1)
         np.add.at(V, (Ellipsis, (b.kc + b.d) % N), b.g * U / b.M)
@@ -401,9 +408,11 @@ def analyse_adjoint(lay: Layout, ybar: Sequence[np.ndarray]) -> np.ndarray:
     return np.conj(long_dft(np.conj(V))).real
 
 
-def synthesise_adjoint(lay: Layout, xbar: np.ndarray) -> List[np.ndarray]:
+def synthesise_adjoint(lay: Layout, xbar: np.ndarray, bands: Optional[Sequence[int]] = None,
+                       n: Optional[Sequence[np.ndarray]] = None) -> List[np.ndarray]:
     """S^dagger xbar: G_k = (w_k/N) [F_N xbar]_k (w = 2, but 1 and real at k = 0, N/2);
-    cbar_lambda = M F_M^{-1} E diag(h) G."""
+    cbar_lambda = M F_M^{-1} E diag(h) G.  With `bands` only those bands are returned; with `n` (one index
+    array per returned band) only those output indices of each."""
     N = lay.N
     xbar = np.asarray(xbar, dtype=np.float64)
     X = long_dft(xbar)
@@ -412,12 +421,14 @@ def synthesise_adjoint(lay: Layout, xbar: np.ndarray) -> List[np.ndarray]:
     G[..., 0] = X[..., 0].real / N
     G[..., N // 2] = X[..., N // 2].real / N
     out = []
-    for b in lay.bands:
+    which = lay.bands if bands is None else [lay.bands[i] for i in bands]
+    for j, b in enumerate(which):
         k = b.kc + b.d
         ok = (k >= 0) & (k <= N // 2)
         vals = b.h[ok] * G[..., k[ok]]
+        nn = np.arange(b.M, dtype=np.int64) if n is None else np.asarray(n[j], dtype=np.int64)
         # M * (1/M) sum_d ... : the two factors cancel
-        out.append(_direct_band_sum(vals, b.d[ok], np.arange(b.M, dtype=np.int64), b.M, +1))
+        out.append(_direct_band_sum(vals, b.d[ok], nn, b.M, +1))
     return out
 
 

@@ -22,8 +22,11 @@ static bool five_smooth(int64_t m) {
 
 int64_t band_length(int64_t S, int policy) {
     int64_t m = 4 * ((S + 3) / 4);
-    if (policy == 0) return m;
-    if (policy == 1) {
+    // Beyond kMaxRaggedLength coefficients a band no longer fits one CTA's shared memory together with the second
+    // buffer a length with a large prime factor needs, and the two-pass kernels take smooth factors only: longer
+    // bands get a 5-smooth length under the multiple-of-4 policy too.
+    if (policy == 0 && m <= kMaxRaggedLength) return m;
+    if (policy == 0 || policy == 1) {
         while (!five_smooth(m)) m += 4;
         return m;
     }

@@ -7,6 +7,10 @@
 
 namespace cqt {
 
+// Longest band the multiple-of-4 policy leaves ragged (see band_length): 2 M + M / 4 complex values must fit the
+// 227 KB of one CTA.
+constexpr int64_t kMaxRaggedLength = 12800;
+
 struct LayoutDesc {
     double fs, fmin, fmax;
     int bins_per_octave;

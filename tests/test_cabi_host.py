@@ -39,6 +39,33 @@ CASES = [wl.CONFIGS["config1"], wl.CONFIGS["config3"], wl.CONFIGS["config5"], wl
          small_workload("pow2", N=4096, fs=8000.0, fmin=100.0, fmax=4000.0, bins_per_octave=24, m_policy=wl.M_POW2)]
 
 
+@pytest.mark.parametrize("name", ["config1", "config2", "config3", "config4", "config5"])
+def test_default_length_policy_plans_every_workload(name):
+    """cqt_plan_create's policy (multiple of 4) on all five workloads: every band gets a radix plan (host-only
+    plans, so no device is needed), lengths up to 12,800 are exactly 4 ceil(S / 4), longer ones are 5-smooth,
+    and the layout agrees with the oracle's."""
+    import dataclasses
+    w = dataclasses.replace(wl.CONFIGS[name], m_policy=wl.M_MULT4)
+    lay = oracle_layout(w)
+    plan = library_plan(w, device=-1)
+    assert plan.num_bands == len(lay.bands) and plan.coeff_count == lay.coeff_count
+    ragged = 0
+    for i, bd in enumerate(lay.bands):
+        bi = plan.band_info(i)
+        assert bi.M == bd.M and bi.M >= bi.support and bi.M % 4 == 0
+        if bi.M <= 12800:
+            assert bi.M == 4 * ((bi.support + 3) // 4)
+            ragged += 1
+        else:
+            m = bi.M
+            for p in (2, 3, 5):
+                while m % p == 0:
+                    m //= p
+            assert m == 1
+    assert ragged >= len(lay.bands) - 120
+    plan.close()
+
+
 @pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
 def test_host_plan_matches_oracle_layout(w):
     lay = oracle_layout(w)

@@ -42,6 +42,62 @@ def test_workload2_round_trip_full_batch():
     plan.close()
 
 
+def test_workload2_under_the_default_length_policy():
+    """Workload 2's layout with the lengths cqt_plan_create picks (multiples of 4: prime factors up to several
+    thousand, chirp-z and direct-sum paths up to 12,800 coefficients, 5-smooth beyond): round trip and sampled
+    coefficients of every third band on two signals."""
+    import dataclasses
+    w = dataclasses.replace(wl.scaled(wl.CONFIGS["config2"], channels=2), m_policy=wl.M_MULT4)
+    lay = oracle_layout(w)
+    plan = library_plan(w)
+    x = wl.make_signal(w)
+    c = plan.analyse(torch.from_numpy(x).cuda(), valid_len=w.valid_len)
+    xr = plan.synthesise(c, valid_len=w.valid_len)
+    assert snr_db(x, xr.cpu().numpy()).min() >= 120.0
+    X = orc.long_dft(orc.pad_signal(x, w.N))
+    worst, band = _sampled_band_errors(lay, X, c.cpu().numpy(), [0, 1], 32, 6, band_step=3)
+    assert worst <= 1e-5, (band, worst)
+    plan.close()
+
+
+def test_longest_single_cta_class_synthesis_and_adjoints():
+    """Workload 2's bands above 13,500 coefficients (the launch class of one 1024-thread CTA per band and signal,
+    up to 216 KB of shared memory): synthesis, T^dagger and S^dagger against the oracle restricted to those bands.
+    The other bands' coefficients are zero, so the oracle's direct sums stay affordable."""
+    w = wl.scaled(wl.CONFIGS["config2"], channels=2)
+    lay = oracle_layout(w)
+    plan = library_plan(w)
+    infos = plan.bands()
+    top = max(bi.launch_class for bi in infos)
+    long_bands = [i for i, bi in enumerate(infos) if bi.launch_class == top]
+    assert len(long_bands) >= 3 and all(13500 < lay.bands[i].M <= 27000 for i in long_bands)
+    rng = np.random.default_rng(41)
+    offs = lay.coeff_offsets
+    y = np.zeros((w.channels, lay.coeff_count), dtype=np.complex64)
+    ysel = []
+    for i in long_bands:
+        M = lay.bands[i].M
+        yb = (rng.standard_normal((w.channels, M)) + 1j * rng.standard_normal((w.channels, M))).astype(np.complex64)
+        y[:, offs[i]:offs[i] + M] = yb
+        ysel.append(yb.astype(np.complex128))
+    yd = torch.from_numpy(y).cuda()
+    got = plan.synthesise(yd, valid_len=w.valid_len).cpu().numpy()
+    want = orc.synthesise(lay, ysel, bands=long_bands)[..., :w.valid_len]
+    assert (np.linalg.norm(got - want, axis=-1) / np.linalg.norm(want, axis=-1)).max() <= 1e-5
+    got = plan.analyse_adjoint(yd, valid_len=w.valid_len).cpu().numpy()
+    want = orc.analyse_adjoint(lay, ysel, bands=long_bands)[..., :w.valid_len]
+    assert (np.linalg.norm(got - want, axis=-1) / np.linalg.norm(want, axis=-1)).max() <= 1e-5
+    # S^dagger: all bands on the GPU, the long ones compared at sampled output indices
+    x = wl.make_signal(w)
+    cb = plan.synthesise_adjoint(torch.from_numpy(x).cuda(), valid_len=w.valid_len).cpu().numpy()
+    ns = [np.unique(np.concatenate([[0, lay.bands[i].M - 1], rng.integers(0, lay.bands[i].M, 64)])) for i in long_bands]
+    want = orc.synthesise_adjoint(lay, orc.pad_signal(x, w.N), bands=long_bands, n=ns)
+    for i, n, wb in zip(long_bands, ns, want):
+        g = cb[:, offs[i] + n]
+        assert (np.linalg.norm(g - wb, axis=-1) / np.linalg.norm(wb, axis=-1)).max() <= 1e-5, i
+    plan.close()
+
+
 def test_workload3_forward_and_adjoint_full_batch():
     w = wl.CONFIGS["config3"]
     lay = oracle_layout(w)

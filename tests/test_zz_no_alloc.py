@@ -24,10 +24,21 @@ def test_static_workspace_analysis_matches_cqt_analyse_twice():
     assert limit == 16 << 20 and plan.workspace_bytes(w.channels) <= limit
     x1 = torch.from_numpy(wl.make_signal(w)).cuda()
     x2 = torch.flip(x1, dims=[1]).contiguous() * 0.5 + 0.25
+    out = torch.empty((w.channels, plan.coeff_count), dtype=torch.complex64, device="cuda")
+    plan.analyse_static_ws(x1, valid_len=w.valid_len, out=out)   # first call on this device: looks the array up
+    torch.cuda.synchronize()
     for x in (x1, x2):
         want = plan.analyse(x, valid_len=w.valid_len)
-        got = plan.analyse_static_ws(x, valid_len=w.valid_len)
         torch.cuda.synchronize()
+        # the call is made for hosts that cannot allocate: with the output preallocated, the device's free
+        # memory is the same before and after it
+        free_before, _ = torch.cuda.mem_get_info()
+        got = plan.analyse_static_ws(x, valid_len=w.valid_len, out=out)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
+        # same kernels, same arguments apart from the scratch pointer: the results are identical bit for bit
+        assert torch.equal(torch.view_as_real(got), torch.view_as_real(want))
         a, b = got.cpu().numpy().astype(np.complex128), want.cpu().numpy().astype(np.complex128)
         o = 0
         for bi in plan.bands():
