@@ -263,7 +263,9 @@ cqt_status cqt_synthesise_adjoint(const cqt_plan *plan, const float *x_bar, int6
  *   slicq_flush  pushes zeros (between sl/2 and sl per channel) up to the next multiple of sl/2 plus sl/2, so
  *                that every frame pushed so far becomes final and can be pulled.
  *   Push, pull and flush of one object must be issued on the same stream (they share staging buffers).
- *   slicq_reset  drops all state and restarts at slice 0 (synchronises the object's stream use).
+ *   slicq_reset  drops all state and restarts at slice 0; waits for the stream of the object's latest push, pull or
+ *                flush (no other stream of the device is synchronised).
+ *   Every slicq call runs on the plan's device and restores the caller's current device.
  */
 cqt_status slicq_create(const cqt_plan *slice_plan, int channels, int64_t transition,
                         int64_t max_slices_in_flight, cqt_slicq **out);

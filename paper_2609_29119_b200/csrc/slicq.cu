@@ -28,9 +28,25 @@ struct cqt_slicq {
     int64_t next_slice = 0;  // first slice not yet analysed
     int64_t next_synth = 0;  // first slice not yet synthesised
     int64_t n_out = 0;       // frames pulled
+    cudaStream_t last_stream = nullptr;   // stream of the latest push / pull / flush (slicq_reset waits for it)
+    bool used = false;
 };
 
 namespace {
+
+// The object's kernels and copies run on the plan's device whatever device the caller has current.
+struct OnPlanDevice {
+    int prev = -1, dev = -1;
+    bool ok = true;
+    explicit OnPlanDevice(const cqt_slicq *s) {
+        dev = s->plan->device;
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~OnPlanDevice() {
+        if (prev >= 0 && prev != dev) cudaSetDevice(prev);
+    }
+};
 
 __global__ void slicq_ingest_kernel(const float *x, long long x_stride, float *ring, long long R, long long pos, long long n, int zero) {
     const int c = blockIdx.y;
@@ -205,6 +221,9 @@ cqt_status slicq_create(const cqt_plan *plan, int channels, int64_t transition, 
 
 cqt_status slicq_push(cqt_slicq *s, const float *x, int64_t x_stride, int64_t n, void *stream, int64_t *slices_completed) {
     if (!s || n < 0 || (n > 0 && (!x || x_stride < n))) return CQT_ERR_INVALID_ARG;
+    OnPlanDevice guard(s);
+    if (!guard.ok) return CQT_ERR_CUDA;
+    if (n > 0) { s->last_stream = reinterpret_cast<cudaStream_t>(stream); s->used = true; }
     cqt_status r = n > 0 ? push_impl(s, x, x_stride, n, 0, reinterpret_cast<cudaStream_t>(stream)) : CQT_OK;
     if (slices_completed) *slices_completed = s->next_slice;
     return r;
@@ -212,6 +231,10 @@ cqt_status slicq_push(cqt_slicq *s, const float *x, int64_t x_stride, int64_t n,
 
 cqt_status slicq_flush(cqt_slicq *s, void *stream) {
     if (!s) return CQT_ERR_INVALID_ARG;
+    OnPlanDevice guard(s);
+    if (!guard.ok) return CQT_ERR_CUDA;
+    s->last_stream = reinterpret_cast<cudaStream_t>(stream);
+    s->used = true;
     // enough zeros that every frame pushed so far becomes final: n_in -> (ceil(n_in / H) + 1) H
     const int64_t target = ((s->n_in + s->H - 1) / s->H + 1) * s->H;
     return push_impl(s, nullptr, 0, target - s->n_in, 1, reinterpret_cast<cudaStream_t>(stream));
@@ -226,7 +249,11 @@ cqt_status slicq_coeffs(cqt_slicq *s, int64_t slice_index, cqt_c64 **c) {
 
 cqt_status slicq_pull(cqt_slicq *s, float *y, int64_t y_stride, int64_t n_max, void *stream, int64_t *n_written) {
     if (!s || n_max < 0 || (n_max > 0 && (!y || y_stride < n_max)) || !n_written) return CQT_ERR_INVALID_ARG;
+    OnPlanDevice guard(s);
+    if (!guard.ok) return CQT_ERR_CUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    s->last_stream = st;
+    s->used = true;
     int64_t written = 0;
     for (;;) {
         // synthesise as many pending slices as the output ring has room for
@@ -263,12 +290,12 @@ cqt_status slicq_pull(cqt_slicq *s, float *y, int64_t y_stride, int64_t n_max, v
 
 cqt_status slicq_reset(cqt_slicq *s) {
     if (!s) return CQT_ERR_INVALID_ARG;
-    int cur = 0;
-    cudaGetDevice(&cur);
-    cudaSetDevice(s->plan->device);
-    cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaMemset(s->d_out, 0, (size_t)s->C * s->ring_out * sizeof(float));
-    cudaSetDevice(cur);
+    OnPlanDevice guard(s);
+    if (!guard.ok) return CQT_ERR_CUDA;
+    // only the stream this object last worked on is waited for, and cleared on: other streams of the device run on
+    cudaError_t e = s->used ? cudaStreamSynchronize(s->last_stream) : cudaSuccess;
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->d_out, 0, (size_t)s->C * s->ring_out * sizeof(float), s->last_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->last_stream);
     s->n_in = s->next_slice = s->next_synth = s->n_out = 0;
     return e == cudaSuccess ? CQT_OK : CQT_ERR_CUDA;
 }
@@ -295,6 +322,8 @@ cqt_status slicq_assemble(cqt_slicq *s, int64_t first_slice, int64_t n_slices, c
     if (!s || !out || n_slices < 1 || first_slice < 0) return CQT_ERR_INVALID_ARG;
     if (out_stride < slicq_assembled_length(s, n_slices)) return CQT_ERR_INVALID_ARG;
     if (first_slice < s->next_synth || first_slice + n_slices > s->next_slice) return CQT_ERR_STATE;
+    OnPlanDevice guard(s);
+    if (!guard.ok) return CQT_ERR_CUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int64_t cc = cqt_plan_coeff_count(s->plan);
     dim3 grid(blocks_for((n_slices + 1) * (cc / 2)), (unsigned)s->C);
@@ -322,6 +351,8 @@ cqt_status slicq_save_state(cqt_slicq *s, void *host_buf, size_t bytes, void *st
     if (!s || !host_buf) return CQT_ERR_INVALID_ARG;
     if (bytes < slicq_state_bytes(s)) return CQT_ERR_WORKSPACE;
     if (s->next_synth != s->next_slice) return CQT_ERR_STATE;    // analysed slices await slicq_pull
+    OnPlanDevice guard(s);
+    if (!guard.ok) return CQT_ERR_CUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     SlicqStateHeader h{kStateMagic, 1u, s->C, 0, s->sl, s->tr, s->K, s->ring_in, s->ring_out, cqt_plan_coeff_count(s->plan),
                        s->n_in, s->next_slice, s->next_synth, s->n_out};
@@ -345,7 +376,11 @@ cqt_status slicq_load_state(cqt_slicq *s, const void *host_buf, size_t bytes, vo
         return CQT_ERR_STATE;                                     // saved by an object of another shape
     if (bytes < slicq_state_bytes(s)) return CQT_ERR_INVALID_ARG;
     if (h.next_synth != h.next_slice || h.n_in < 0 || h.n_out < 0 || h.n_out > h.n_in) return CQT_ERR_INVALID_ARG;
+    OnPlanDevice guard(s);
+    if (!guard.ok) return CQT_ERR_CUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    s->last_stream = st;
+    s->used = true;
     const char *p = static_cast<const char *>(host_buf);
     const size_t b_in = (size_t)s->C * s->ring_in * sizeof(float), b_out = (size_t)s->C * s->ring_out * sizeof(float);
     cudaError_t e = cudaMemcpyAsync(s->d_in, p + sizeof h, b_in, cudaMemcpyHostToDevice, st);
