@@ -584,6 +584,9 @@ def run_sweep(args, w):
     torch.cuda.set_device(0)
     plan = make_plan(w, 0)
     batches = [args.channels] if args.channels else sorted(PAPER_A100_MS)
+    if not args.no_torchfft:
+        from torchfft_baseline import TorchFftCqt
+        tf = TorchFftCqt(plan, torch.device("cuda:0"))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # larger than the 126 MB L2
     stream = torch.cuda.current_stream()
     K = min(args.steps, 50)
@@ -630,12 +633,26 @@ def run_sweep(args, w):
         graph = capture_graph(step)
         hot = median_ms(graph.replay, False)
         cold = median_ms(graph.replay, True)
+        # same-box comparator (the paper's "CQT baseline": the operator through torch.fft / cuFFT calls)
+        tf_res = {}
+        if not args.no_torchfft:
+            def tf_step(st=None):
+                tf.synthesise(tf.analyse(x))
+            tf_y = tf.synthesise(tf.analyse(x))
+            xd0, yd0 = x.double(), tf_y.double()
+            tf_snr = float((10 * torch.log10((xd0 * xd0).sum(1) / ((xd0 - yd0) ** 2).sum(1))).min())
+            tf_eager = median_ms(tf_step, False)
+            tf_graph = capture_graph(tf_step)
+            tf_hot = median_ms(tf_graph.replay, False)
+            del tf_graph
+            tf_res = {"torchfft_eager_ms": tf_eager, "torchfft_graph_ms": tf_hot, "torchfft_snr_db_min": tf_snr,
+                      "speedup_vs_torchfft_graph": tf_hot / hot, "speedup_vs_torchfft_eager": tf_eager / eager}
         xd, xrd = x.double(), xr.double()
         snr = float((10 * torch.log10((xd * xd).sum(1) / ((xd - xrd) ** 2).sum(1))).min())
         sweep[str(B)] = {"eager_ms": eager, "graph_ms": hot, "graph_l2_flushed_ms": cold, "snr_db_min": snr,
                          "paper_a100_graph_ms": PAPER_A100_MS.get(B),
                          "step_with_backward_eager_ms": backward, "paper_a100_backward_ms": PAPER_A100_BACKWARD_MS.get(B), "workspace_mb_per_signal": plan.workspace_bytes(B) / B / 1e6,
-                         "msamples_per_s_l2_flushed": B * w.valid_len / cold / 1e3}
+                         "msamples_per_s_l2_flushed": B * w.valid_len / cold / 1e3, **tf_res}
         del graph
     launches = plan.launch_count() - launches0
     clocks = sampler.stop()
@@ -677,6 +694,7 @@ def main():
     ap.add_argument("--min-seconds", type=float, default=0.5,
                     help="repeat the timed region of --steps steps until this much device time has passed")
     ap.add_argument("--no-secondary", action="store_true", help="skip the second batched workload (config3)")
+    ap.add_argument("--no-torchfft", action="store_true", help="table1 sweep: skip the torch.fft comparator")
     ap.add_argument("--tune", action="append", default=[], metavar="FIELD=VALUE",
                     help="a field of cqt_plan_tuning (max_cta_elems, two_pass_min); "
                          "the defaults are what the library ships with")
