@@ -39,7 +39,7 @@ static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, Ba
     void *args[] = {&a};
     const void *fn = class_kernel<ANALYSIS>(c);
     if (!fn) return cudaErrorInvalidDeviceFunction;
-    cudaError_t e = cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(c.threads), args, smem, st);
+    cudaError_t e = launch_kernel(fn, dim3((unsigned)grid), dim3(c.threads), args, smem, st);
     note_launch(p, name, st);
     return e;
 }

@@ -26,6 +26,7 @@ struct RegularStore {
 
 template <int THREADS, int MINB, bool WARP, int MAXR, bool GEN>
 __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandArgs a) {
+    pdl_launch_dependents();
     using G = Group<WARP>;
     using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
     const int item = G::item();
@@ -34,6 +35,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     __shared__ BandItem item_s[WARP ? 8 : 1];
     BandItem &it = item_s[G::slot()];
     fetch_item<Sync>(a.items[a.work[item / a.batch]], it, tid, nthr);
+    pdl_wait();   // record and plan belong to the plan; everything below touches the predecessor's output
     const BandRec br = it.br;
     const int ch = item % a.batch;
     const FftPlan &fp = it.fp;

@@ -12,6 +12,14 @@
 
 namespace cqt {
 
+// Programmatic dependent launch (sm_90 and later): a kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream is still running.  Every kernel of the library lets its successor start
+// early (pdl_launch_dependents at its top) and waits for its predecessor (pdl_wait) only after the prologue that reads
+// nothing but the plan's tables (band record, radix plan, twiddle tables): launch latency and that prologue overlap
+// the predecessor's tail.  Without the attribute both calls do nothing.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 struct BlockSync {
     static __device__ __forceinline__ void sync() { __syncthreads(); }
 };

@@ -117,6 +117,21 @@ inline cudaError_t allow_dynamic_smem(const void *fn, size_t need, const cqt_pla
 
 cudaError_t configure_long_fft_kernels(const cqt_plan &p);
 
+// Launch with the programmatic-serialization attribute (see pdl_wait in engine.cuh).
+inline cudaError_t launch_kernel(const void *fn, dim3 grid, dim3 block, void **args, size_t smem, cudaStream_t st) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelExC(&cfg, fn, args);
+}
+
 // band.cu
 cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
                                        int64_t batch, cudaStream_t st);

@@ -125,6 +125,7 @@ __device__ __forceinline__ void cols_fwd_body(const LongArgs &a, const FftPlan &
 
 template <class SH>
 __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
     const int j2_0 = blockIdx.x * TW;
@@ -135,6 +136,7 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     float2 *wl = tws + fp.M;
     stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
+    pdl_wait();   // the tables above belong to the plan; what follows reads the predecessor's output
     cols_fwd_body<SH>(a, fp, buf, tws, wl, j2_0, ch, tid, nthr);
 }
 
@@ -208,6 +210,7 @@ __device__ __forceinline__ void rows_fwd_body(const LongArgs &a, const FftPlan &
 
 template <class SH>
 __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
     const bool direct = (a.A == 1);
@@ -219,6 +222,7 @@ __global__ void __launch_bounds__(512, 2) rfft_rows_fwd_kernel(LongArgs a) {
     float2 *wn = tws + fp.M;
     stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
+    pdl_wait();   // the tables above belong to the plan; what follows reads the predecessor's output
     rows_fwd_body<SH>(a, fp, buf, tws, wn, t, ch, tid, nthr);
 }
 
@@ -393,6 +397,7 @@ __device__ __forceinline__ void rows_inv_body(const LongArgs &a, const FftPlan &
 
 template <class SH>
 __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int ch = blockIdx.y, t = blockIdx.x;
     const bool direct = (a.A == 1);
@@ -406,6 +411,7 @@ __global__ void __launch_bounds__(512, 2) irfft_rows_kernel(LongArgs a) {
     stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wn, a.tw + a.tw_n, a.n_n, tid, nthr);
     if (!direct) stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
+    pdl_wait();   // the tables above belong to the plan; what follows reads the predecessor's output
     rows_inv_body<SH>(a, fp, buf, tws, wl, wn, t, ch, tid, nthr);
 }
 
@@ -432,6 +438,7 @@ __device__ __forceinline__ void cols_inv_body(const LongArgs &a, const FftPlan &
 
 template <class SH>
 __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int TW = a.tw_cols;
     const int j2_0 = blockIdx.x * TW;
@@ -440,6 +447,7 @@ __global__ void __launch_bounds__(512, 2) irfft_cols_kernel(LongArgs a) {
     float2 *buf = smem_long;
     float2 *tws = buf + (size_t)a.A * (TW | 1);
     stage_full(tws, a.tw, fp, tid, nthr);
+    pdl_wait();   // the tables above belong to the plan; what follows reads the predecessor's output
     cols_inv_body<SH>(a, fp, buf, tws, j2_0, ch, tid, nthr);
 }
 
@@ -535,7 +543,7 @@ static const void *cols_inv_fn(const cqt_plan &p) {
 }
 static cudaError_t launch_long(const void *fn, dim3 grid, int threads, size_t smem, LongArgs &a, cudaStream_t st) {
     void *args[] = {&a};
-    return cudaLaunchKernel(fn, grid, dim3((unsigned)threads), args, smem, st);
+    return launch_kernel(fn, grid, dim3((unsigned)threads), args, smem, st);
 }
 
 static int threads_for(size_t butterflies) {
