@@ -65,6 +65,7 @@ __device__ __forceinline__ void copy_table(float2 *dst, const float2 *__restrict
 // pass 1: kTW adjacent columns (second index), A-point transform over the first index, inter-pass twiddle
 template <int THREADS, int MINB, bool ANALYSIS>
 __global__ void __launch_bounds__(THREADS, MINB) band2p_cols_kernel(TwoPassArgs a) {
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const TwoPassRec rec = a.recs[blockIdx.y / a.groups];
     const int ch0 = (blockIdx.y % a.groups) * a.ch_per_cta, ch1 = min(a.batch, ch0 + a.ch_per_cta);
@@ -81,6 +82,7 @@ __global__ void __launch_bounds__(THREADS, MINB) band2p_cols_kernel(TwoPassArgs 
     const float *tab = a.table + br.tab_off;
     const bool fold = !ANALYSIS && a.fold && br.side != 0;
     const Tile t{buf, kTW, kTW, 1u << 28, rec.A * kTW, a.dbg};
+    pdl_wait();   // tables and records belong to the plan; the loop touches the predecessor's output
     for (int ch = ch0; ch < ch1; ++ch) {
     const float2 *X = ANALYSIS ? a.spec + (long long)ch * a.spec_pitch : nullptr;
     const float2 *cin = ANALYSIS ? nullptr : a.coef + (long long)ch * a.coeff_count + br.coeff_off;
@@ -107,6 +109,7 @@ __global__ void __launch_bounds__(THREADS, MINB) band2p_cols_kernel(TwoPassArgs 
 // pass 2: kTW adjacent rows (first output index), B-point transform over the second index
 template <int THREADS, int MINB, bool ANALYSIS>
 __global__ void __launch_bounds__(THREADS, MINB) band2p_rows_kernel(TwoPassArgs a) {
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const TwoPassRec rec = a.recs[blockIdx.y / a.groups];
     const int ch0 = (blockIdx.y % a.groups) * a.ch_per_cta, ch1 = min(a.batch, ch0 + a.ch_per_cta);
@@ -120,6 +123,7 @@ __global__ void __launch_bounds__(THREADS, MINB) band2p_rows_kernel(TwoPassArgs 
     float2 *twf = buf + (size_t)rec.B * pitch;
     copy_table(twf, a.tw + fp.tw_full_off, rec.B, tid, nthr);
     const Tile t{buf, pitch, kTW, 1u << 28, rec.B * pitch, a.dbg};
+    pdl_wait();   // tables and records belong to the plan; the loop touches the predecessor's output
     for (int ch = ch0; ch < ch1; ++ch) {
     const float2 *T = a.scratch + (long long)ch * a.scratch_pitch + rec.scratch_off;
     auto load = [&](int p, int r) -> float2 {
@@ -197,11 +201,11 @@ static cudaError_t run_group(const cqt_plan &p, int g, const float *table, bool 
     a.groups = (int)((batch + cpc - 1) / cpc);
     void *args[] = {&a};
     dim3 g1((unsigned)grp.max_tiles_cols, (unsigned)(grp.bands.size() * a.groups));
-    cudaError_t e = cudaLaunchKernel(cols_kernel<ANALYSIS>(g), g1, dim3(threads), args, grp.smem_cols, st);
+    cudaError_t e = launch_kernel(cols_kernel<ANALYSIS>(g), g1, dim3(threads), args, grp.smem_cols, st);
     note_launch(p, ANALYSIS ? (g ? "band2p_cols/analysis/large" : "band2p_cols/analysis") : (g ? "band2p_cols/synthesis/large" : "band2p_cols/synthesis"), st);
     if (e != cudaSuccess) return e;
     dim3 g2((unsigned)grp.max_tiles_rows, (unsigned)(grp.bands.size() * a.groups));
-    e = cudaLaunchKernel(rows_kernel<ANALYSIS>(g), g2, dim3(threads), args, grp.smem_rows, st);
+    e = launch_kernel(rows_kernel<ANALYSIS>(g), g2, dim3(threads), args, grp.smem_rows, st);
     note_launch(p, ANALYSIS ? (g ? "band2p_rows/analysis/large" : "band2p_rows/analysis") : (g ? "band2p_rows/synthesis/large" : "band2p_rows/synthesis"), st);
     return e;
 }

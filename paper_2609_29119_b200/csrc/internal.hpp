@@ -132,6 +132,22 @@ inline cudaError_t launch_kernel(const void *fn, dim3 grid, dim3 block, void **a
     return cudaLaunchKernelExC(&cfg, fn, args);
 }
 
+// The same for a kernel called with its arguments (replaces kernel<<<grid, block, smem, st>>>(args...)).
+template <class... KArgs, class... Args>
+inline cudaError_t launch_kernel_args(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // band.cu
 cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
                                        int64_t batch, cudaStream_t st);

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "../../include/cqt.h"
+#include "engine.cuh"
 #include "internal.hpp"
 
 struct cqt_slicq {
@@ -49,6 +50,8 @@ struct OnPlanDevice {
 };
 
 __global__ void slicq_ingest_kernel(const float *x, long long x_stride, float *ring, long long R, long long pos, long long n, int zero) {
+    cqt::pdl_launch_dependents();
+    cqt::pdl_wait();
     const int c = blockIdx.y;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         ring[c * R + (pos + i) % R] = zero ? 0.f : x[c * x_stride + i];
@@ -57,6 +60,8 @@ __global__ void slicq_ingest_kernel(const float *x, long long x_stride, float *r
 // stage[(s - s0) * C + c][i] = w[i] * stream[c][s H - H + i]  (zero before the start of the stream)
 __global__ void slicq_cut_kernel(const float *ring, long long R, const float *w, float *stage, long long sl, long long H,
                                  long long s0, int C) {
+    cqt::pdl_launch_dependents();
+    cqt::pdl_wait();
     const long long s = s0 + blockIdx.y / C;
     const int c = blockIdx.y % C;
     float *dst = stage + (long long)blockIdx.y * sl;
@@ -72,6 +77,8 @@ __global__ void slicq_cut_kernel(const float *ring, long long R, const float *w,
 //                         + first half of slice b + 1 (when b + 1 <= s1).
 __global__ void slicq_ola_kernel(const float *stage, float *ring, long long R, long long sl, long long H, long long s0,
                                  long long s1, int C) {
+    cqt::pdl_launch_dependents();
+    cqt::pdl_wait();
     const int c = blockIdx.y;
     const long long lo = (s0 - 1) * H, hi = (s1 + 1) * H;
     for (long long n = lo + blockIdx.x * (long long)blockDim.x + threadIdx.x; n < hi; n += (long long)gridDim.x * blockDim.x) {
@@ -84,6 +91,8 @@ __global__ void slicq_ola_kernel(const float *stage, float *ring, long long R, l
 }
 
 __global__ void slicq_emit_kernel(const float *ring, long long R, long long pos, float *y, long long y_stride, long long n) {
+    cqt::pdl_launch_dependents();
+    cqt::pdl_wait();
     const int c = blockIdx.y;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         y[c * y_stride + i] = ring[c * R + (pos + i) % R];
@@ -128,8 +137,9 @@ cqt_status analyse_ready(cqt_slicq *s, cudaStream_t st) {
         const int64_t slot = s->next_slice % s->K;
         const int64_t cnt = std::min<int64_t>(ready - s->next_slice, s->K - slot);
         dim3 grid(blocks_for(s->sl), (unsigned)(cnt * s->C));
-        slicq_cut_kernel<<<grid, 256, 0, st>>>(s->d_in, s->ring_in, s->d_win, s->d_stage, s->sl, s->H, s->next_slice, s->C);
-        if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+        if (cqt::launch_kernel_args(slicq_cut_kernel, grid, dim3(256), 0, st, s->d_in, s->ring_in, s->d_win, s->d_stage, s->sl, s->H,
+                               s->next_slice, s->C) != cudaSuccess)
+            return CQT_ERR_CUDA;
         cqt_status r = cqt_analyse(s->plan, s->d_stage, s->sl, cnt * s->C, s->sl,
                                    s->d_coef + slot * s->C * cqt_plan_coeff_count(s->plan), s->d_ws, s->ws_bytes, st);
         if (r != CQT_OK) return r;
@@ -150,8 +160,9 @@ cqt_status push_impl(cqt_slicq *s, const float *x, int64_t x_stride, int64_t n, 
         const int64_t m = std::min<int64_t>(n - done, room);
         if (m <= 0) return CQT_ERR_STATE;
         dim3 grid(blocks_for(m), (unsigned)s->C);
-        slicq_ingest_kernel<<<grid, 256, 0, st>>>(zero ? nullptr : x + done, x_stride, s->d_in, s->ring_in, s->n_in, m, zero);
-        if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+        if (cqt::launch_kernel_args(slicq_ingest_kernel, grid, dim3(256), 0, st, zero ? (const float *)nullptr : x + done, x_stride, s->d_in,
+                               s->ring_in, s->n_in, m, zero) != cudaSuccess)
+            return CQT_ERR_CUDA;
         s->n_in += m;
         done += m;
         cqt_status r = analyse_ready(s, st);
@@ -267,9 +278,9 @@ cqt_status slicq_pull(cqt_slicq *s, float *y, int64_t y_stride, int64_t n_max, v
                                           s->d_stage, s->sl, s->d_ws, s->ws_bytes, st);
             if (r != CQT_OK) return r;
             dim3 grid(blocks_for((cnt + 1) * s->H), (unsigned)s->C);
-            slicq_ola_kernel<<<grid, 256, 0, st>>>(s->d_stage, s->d_out, s->ring_out, s->sl, s->H, s->next_synth,
-                                                   s->next_synth + cnt - 1, s->C);
-            if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+            if (cqt::launch_kernel_args(slicq_ola_kernel, grid, dim3(256), 0, st, s->d_stage, s->d_out, s->ring_out, s->sl, s->H,
+                                   s->next_synth, s->next_synth + cnt - 1, s->C) != cudaSuccess)
+                return CQT_ERR_CUDA;
             s->next_synth += cnt;
         }
         // frames below (next_synth - 1) H are final
@@ -277,8 +288,9 @@ cqt_status slicq_pull(cqt_slicq *s, float *y, int64_t y_stride, int64_t n_max, v
         const int64_t m = std::min<int64_t>(n_max - written, final_to - s->n_out);
         if (m > 0) {
             dim3 grid(blocks_for(m), (unsigned)s->C);
-            slicq_emit_kernel<<<grid, 256, 0, st>>>(s->d_out, s->ring_out, s->n_out, y + written, y_stride, m);
-            if (cudaGetLastError() != cudaSuccess) return CQT_ERR_CUDA;
+            if (cqt::launch_kernel_args(slicq_emit_kernel, grid, dim3(256), 0, st, s->d_out, s->ring_out, s->n_out, y + written, y_stride,
+                                   m) != cudaSuccess)
+                return CQT_ERR_CUDA;
             s->n_out += m;
             written += m;
         }
