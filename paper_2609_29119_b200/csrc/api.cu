@@ -176,11 +176,11 @@ void free_device(cqt_plan *p) {
     int cur = 0;
     cudaGetDevice(&cur);
     cudaSetDevice(p->device);
-    cudaFree(p->d.bands); cudaFree(p->d.items); cudaFree(p->d.ffts); cudaFree(p->d.tw);
+    cudaFree(p->d.bands); cudaFree(p->d.ffts); cudaFree(p->d.tw);
     cudaFree(p->d.tab_analysis); cudaFree(p->d.tab_synthesis);
     cudaFree(p->d.tab_analysis_adj); cudaFree(p->d.tab_synthesis_adj);
     cudaFree(p->d.cover); cudaFree(p->d.dbg); cudaFree(p->d.zero_seg);
-    for (auto &c : p->cls) cudaFree(c.d_work);
+    for (auto &c : p->cls) cudaFree(c.d_items);
     for (auto &g : p->two_pass) cudaFree(g.d_recs);
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     for (int i = 0; i < 2; ++i) {
@@ -459,15 +459,6 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
     cudaError_t e = cudaSuccess;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
     chk(upload(p->d.bands, p->bands));
-    {
-        std::vector<BandItem> items(p->bands.size());
-        for (size_t i = 0; i < items.size(); ++i) {
-            items[i].br = p->bands[i];
-            if (p->bands[i].fft >= 0) items[i].fp = p->ffts[(size_t)p->bands[i].fft];
-            else std::memset(&items[i].fp, 0, sizeof(FftPlan));
-        }
-        chk(upload(p->d.items, items));
-    }
     chk(upload(p->d.ffts, p->ffts));
     chk(upload(p->d.tw, tw));
     chk(upload(p->d.tab_analysis, tA));
@@ -486,7 +477,16 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
     p->n_zero_seg = (int)zero_seg.size();
     if (p->n_zero_seg) chk(upload(p->d.zero_seg, zero_seg));
     chk(upload(p->d.dbg, std::vector<int>(8, 0)));
-    for (auto &c : p->cls) chk(upload(c.d_work, c.work));
+    for (auto &c : p->cls) {
+        // record and radix plan of every band of the class, in launch order: what a work item fetches first
+        std::vector<BandItem> items(c.work.size());
+        for (size_t i = 0; i < items.size(); ++i) {
+            const int b = c.work[i];
+            items[i].br = p->bands[(size_t)b];
+            items[i].fp = p->ffts[(size_t)p->bands[(size_t)b].fft];
+        }
+        chk(upload(c.d_items, items));
+    }
     cudaDeviceProp prop;
     chk(cudaGetDeviceProperties(&prop, p->device));
     p->sm_count = prop.multiProcessorCount;

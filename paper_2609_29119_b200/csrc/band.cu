@@ -5,11 +5,10 @@ namespace cqt {
 
 static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *table, int64_t batch) {
     BandArgs a{};
-    a.items = p.d.items;
+    a.items = c.d_items;
     a.ffts = p.d.ffts;
     a.tw = p.d.tw;
     a.table = table;
-    a.work = c.d_work;
     a.n_work = c.n_bands;
     a.batch = (int)batch;
     a.N = (int)p.N;

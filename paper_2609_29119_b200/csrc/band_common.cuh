@@ -16,11 +16,10 @@
 namespace cqt {
 
 struct BandArgs {
-    const BandItem *items;   // per band: record + radix plan
+    const BandItem *items;   // per band of the class, in launch order (longest first): record + radix plan
     const FftPlan *ffts;
     const float2 *tw;
     const float *table;
-    const int32_t *work;     // band indices of this class, longest first
     int n_work;
     int batch;
     int N;

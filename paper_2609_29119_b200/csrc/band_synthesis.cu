@@ -34,8 +34,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     const int tid = G::tid(), nthr = G::nthr();
     __shared__ BandItem item_s[WARP ? 8 : 1];
     BandItem &it = item_s[G::slot()];
-    fetch_item<Sync>(a.items[a.work[item / a.batch]], it, tid, nthr);
-    pdl_wait();   // record and plan belong to the plan; everything below touches the predecessor's output
+    fetch_item<Sync>(a.items[item / a.batch], it, tid, nthr);   // records in launch order of the class
     const BandRec br = it.br;
     const int ch = item % a.batch;
     const FftPlan &fp = it.fp;
@@ -68,6 +67,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     };
     // GEN: the class holds lengths with prime factors above 5 (only the multiple-of-4 length policy makes them);
     // the other instantiations leave the chirp-z and direct-sum code out
+    if (GEN && fp.generic) pdl_wait();
     if (GEN && fp.generic == 2) {
         chirp_z_transform<-1, Sync>(buf, fp, a.ffts, a.tw, load, store, a.dbg, tid, nthr);
         return;
@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_to_spectrum_kernel(BandAr
     }
     float2 *tws = buf + M + 16;
     if (fp.nstages > 1) stage_twiddles(tws, a.tw, fp, tid, nthr);
+    pdl_wait();   // record, plan and twiddle table belong to the plan; what follows touches the predecessor's output
     const Tile t{buf, 1, 1, 0u, M + 16, a.dbg};
     if (br.side == 0) {
         // regular band: all bins in range, plane row and table share the support index j = d - d0

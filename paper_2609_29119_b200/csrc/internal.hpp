@@ -21,7 +21,7 @@ struct BandClass {
     bool has_generic = false; // some band of the class has a prime factor above 5 (direct-sum stage or chirp-z)
     int max_elems = 0;       // shared-memory elements (float2) per item
     int n_bands = 0;         // bands in the class
-    int32_t *d_work = nullptr;  // band indices, longest first
+    BandItem *d_items = nullptr;   // records + radix plans of the class's bands, longest first
     std::vector<int32_t> work;
 };
 
@@ -47,7 +47,6 @@ struct TwoPassGroup {
 
 struct DevicePlan {
     BandRec *bands = nullptr;
-    BandItem *items = nullptr;         // per band: record + plan (plan zeroed for bands on the two-pass kernels)
     FftPlan *ffts = nullptr;
     float2 *tw = nullptr;
     float *tab_analysis = nullptr;     // g / M
