@@ -477,6 +477,17 @@ def run_ours(args, w):
     secondary = None
     if world == 1 and w.name == "config2" and not args.channels and not args.no_secondary:
         secondary = measure_secondary(args, local)
+    cufft = None
+    if world == 1 and not args.no_cufft_calibration:
+        # the vendor FFT alone on the same transform sizes (no windowing, gather or overlap-add): context for the
+        # per-kernel times above, never part of `value`
+        try:
+            from torchfft_baseline import cufft_same_shape_times
+            cufft = cufft_same_shape_times(plan, batch, dev)
+            cufft["unit"] = "us"
+            cufft["step_over_fft_calls_only"] = (ms / K * 1e3) / cufft["round_trip_fft_calls_only"]
+        except Exception as e:  # a calibration aid must never take the bench line down
+            cufft = {"error": f"{type(e).__name__}: {e}"}
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         s = oracle_sample(w, budget_macs=args.cpu_budget_macs)
@@ -516,6 +527,7 @@ def run_ours(args, w):
                          "flops_per_step": path_algorithmic_flops(plan, w, batch)},
         "kernels": kernels,
         "secondary": secondary,
+        "cufft_same_shape": cufft,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
@@ -694,6 +706,8 @@ def main():
     ap.add_argument("--min-seconds", type=float, default=0.5,
                     help="repeat the timed region of --steps steps until this much device time has passed")
     ap.add_argument("--no-secondary", action="store_true", help="skip the second batched workload (config3)")
+    ap.add_argument("--no-cufft-calibration", action="store_true",
+                    help="skip timing the vendor FFT alone on the step's transform sizes")
     ap.add_argument("--no-torchfft", action="store_true", help="table1 sweep: skip the torch.fft comparator")
     ap.add_argument("--tune", action="append", default=[], metavar="FIELD=VALUE",
                     help="a field of cqt_plan_tuning (max_cta_elems, two_pass_min); "

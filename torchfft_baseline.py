@@ -81,3 +81,85 @@ class TorchFftCqt:
         Xh[:, 0] = Xh[:, 0].real.to(torch.complex64)
         Xh[:, -1] = Xh[:, -1].real.to(torch.complex64)
         return torch.fft.irfft(Xh, n=self.N)
+
+
+def _smooth_at_least(n: int) -> int:
+    """Smallest length 2^a 3^b 5^c >= n."""
+    best = None
+    p2 = 1
+    while p2 < 2 * n:
+        p3 = p2
+        while p3 < 2 * n:
+            p5 = p3
+            while p5 < 2 * n:
+                if p5 >= n and (best is None or p5 < best):
+                    best = p5
+                p5 *= 5
+            p3 *= 3
+        p2 *= 2
+    return best
+
+
+def cufft_same_shape_times(plan, batch, device, class_limits=(128, 1024, 4096, 13500), iters=20, warmup=5):
+    """Calibration: what the vendor FFT needs for transforms of the round trip's sizes alone.
+
+    One `torch.fft.rfft` / `irfft` of the batch at the plan's signal length, and per band-length class ONE batched
+    complex transform of (bands in the class x batch) rows at the 5-smooth length nearest above the class's mean
+    band length, so that each call moves the element count of the class within a few percent.  No windowing,
+    gather, zero fill, overlap-add or ragged lengths: this is a lower bound of what a pipeline assembled from
+    library FFTs spends inside the FFT calls, measured with CUDA events on the current stream, three rotating
+    inputs (together larger than the L2 at the headline size).  Returns microseconds per call.
+    """
+    import torch
+
+    def timed(fn):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize(device)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize(device)
+        return a.elapsed_time(b) / iters * 1e3
+
+    out = {}
+    turn = [0]
+    xs = [torch.randn(batch, plan.N, device=device) for _ in range(3)]
+
+    def fwd():
+        turn[0] += 1
+        return torch.fft.rfft(xs[turn[0] % 3])
+    out["rfft"] = timed(fwd)
+    Xs = [torch.fft.rfft(x) for x in xs]
+    del xs
+
+    def inv():
+        turn[0] += 1
+        return torch.fft.irfft(Xs[turn[0] % 3], n=plan.N)
+    out["irfft"] = timed(inv)
+    del Xs
+    lengths = [int(b.M) for b in plan.bands()]
+    lo = 0
+    classes = {}
+    for ci, hi in enumerate(list(class_limits) + [max(lengths) + 1]):
+        mine = [m for m in lengths if lo < m <= hi]
+        lo = hi
+        if not mine:
+            continue
+        M = _smooth_at_least(-(-sum(mine) // len(mine)))
+        rows = len(mine) * batch
+        cs = [torch.randn(rows, M, dtype=torch.complex64, device=device) for _ in range(3)]
+        dst = torch.empty_like(cs[0])
+
+        def c2c():
+            turn[0] += 1
+            torch.fft.fft(cs[turn[0] % 3], out=dst)
+        classes[f"class{ci}"] = {"rows": rows, "length": M, "elements_vs_class": rows * M / (sum(mine) * batch),
+                                 "us": timed(c2c)}
+        del cs, dst
+    out["classes"] = classes
+    out["band_ffts_one_direction"] = sum(c["us"] for c in classes.values())
+    out["round_trip_fft_calls_only"] = out["rfft"] + out["irfft"] + 2 * out["band_ffts_one_direction"]
+    return out
