@@ -436,6 +436,23 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
             g.smem_rows = std::max(g.smem_rows, two_pass_smem_rows(tb));
         }
     }
+    // estimates for the per-call assignment of classes to streams (band.cu): total work, and the time one CTA
+    // needs for the longest item (microseconds per element by class, from measured kernel times)
+    {
+        const double us_per_elem[kNumClasses] = {0.04, 0.015, 0.004, 0.0016, 0.0016};
+        // classes holding lengths with a prime factor above 5 (direct sums, chirp-z with two longer transforms)
+        const double generic_factor[kNumClasses] = {1.3, 1.3, 2.0, 3.5, 3.5};
+        for (int c = 0; c < kNumClasses; ++c) {
+            BandClass &bc = p->cls[c];
+            int64_t longest = 0;
+            for (int32_t b : bc.work) {
+                const int64_t M = p->bands[(size_t)b].M;
+                bc.stage_work += (double)M * (p->ffts[(size_t)p->bands[(size_t)b].fft].nstages + 1);
+                longest = std::max(longest, M);
+            }
+            bc.latency_us = bc.n_bands ? (5.0 + us_per_elem[c] * (double)longest) * (bc.has_generic ? generic_factor[c] : 1.0) : 0.0;
+        }
+    }
     if (p->device < 0) { *out = p; return CQT_OK; }
 
     // ---- device tables

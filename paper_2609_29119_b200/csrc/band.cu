@@ -1,4 +1,6 @@
 // Host side of the fused band kernels: per-class launches on the caller's stream and the plan's helper streams.
+#include <algorithm>
+
 #include "band_common.cuh"
 
 namespace cqt {
@@ -43,22 +45,43 @@ static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, Ba
     return e;
 }
 
-// The classes of one call are independent (disjoint outputs), and the short-band classes alone leave most SMs
-// idle, so they run on two helper streams beside the long-band classes: fork after the caller's stream, join
-// back into it.  With event timing on, everything stays on the caller's stream.
+// The classes of one call are independent (disjoint outputs), and most of them alone leave SMs idle, so they run
+// side by side on the caller's stream and two helper streams: fork after the caller's stream, join back into it.
+// Per call, each class's run time is estimated as the larger of the time of its longest work item and its work
+// at this batch size over the machine's throughput; the classes go, longest first, to the stream with the least
+// time so far (the longest one therefore stays on the caller's stream).  With event timing on, everything stays
+// on the caller's stream.
 struct ForkJoin {
     const cqt_plan &p;
     cudaStream_t st;
     bool used[2] = {false, false};
     bool serial;
-    ForkJoin(const cqt_plan &plan, cudaStream_t s) : p(plan), st(s), serial(plan.timing || !plan.aux[0] || !plan.aux[1]) {
-        if (!serial) cudaEventRecord(p.ev_fork, st);
+    int slot[kNumClasses] = {0, 0, 0, 0, 0};
+    ForkJoin(const cqt_plan &plan, cudaStream_t s, int64_t batch)
+        : p(plan), st(s), serial(plan.timing || !plan.aux[0] || !plan.aux[1]) {
+        if (serial) return;
+        constexpr double kElementStagesPerUs = 6.7e5;   // the 4096 < M <= 13,500 class at 32 signals
+        double est[kNumClasses], load[3] = {0.0, 0.0, 0.0};
+        int order[kNumClasses];
+        for (int c = 0; c < kNumClasses; ++c) {
+            order[c] = c;
+            est[c] = p.cls[c].n_bands ? std::max(p.cls[c].latency_us, p.cls[c].stage_work * (double)batch / kElementStagesPerUs) : 0.0;
+        }
+        std::stable_sort(order, order + kNumClasses, [&](int a, int b) { return est[a] > est[b]; });
+        for (int i = 0; i < kNumClasses; ++i) {
+            const int c = order[i];
+            if (!p.cls[c].n_bands) continue;
+            int best = 0;
+            for (int j = 1; j < 3; ++j)
+                if (load[j] < load[best]) best = j;
+            slot[c] = best;
+            load[best] += est[c];
+        }
+        cudaEventRecord(p.ev_fork, st);
     }
     cudaStream_t stream_for(int cls) {
-        if (serial || cls == 3 || p.cls[cls].n_bands == 0) return st;
-        // the longest bands (one CTA per SM, fewer CTAs than SMs) and the middle class share one helper stream,
-        // the two short classes the other; the 4096 < M <= 13,500 class stays on the caller's stream
-        const int i = (cls == 2 || cls == 4) ? 0 : 1;
+        if (serial || slot[cls] == 0 || p.cls[cls].n_bands == 0) return st;
+        const int i = slot[cls] - 1;
         if (!used[i]) { cudaStreamWaitEvent(p.aux[i], p.ev_fork, 0); used[i] = true; }
         return p.aux[i];
     }
@@ -70,7 +93,7 @@ struct ForkJoin {
 
 cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
                                        int64_t batch, cudaStream_t st) {
-    ForkJoin fj(p, st);
+    ForkJoin fj(p, st, batch);
     static const char *names[kNumClasses] = {"bands_from_spectrum/class0", "bands_from_spectrum/class1",
                                               "bands_from_spectrum/class2", "bands_from_spectrum/class3",
                                               "bands_from_spectrum/class4"};
@@ -101,7 +124,7 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    ForkJoin fj(p, st);
+    ForkJoin fj(p, st, batch);
     static const char *names[kNumClasses] = {"bands_to_spectrum/class0", "bands_to_spectrum/class1",
                                               "bands_to_spectrum/class2", "bands_to_spectrum/class3",
                                               "bands_to_spectrum/class4"};

@@ -21,6 +21,8 @@ struct BandClass {
     bool has_generic = false; // some band of the class has a prime factor above 5 (direct-sum stage or chirp-z)
     int max_elems = 0;       // shared-memory elements (float2) per item
     int n_bands = 0;         // bands in the class
+    double stage_work = 0.0; // element-stages of the class's transforms per signal (stream assignment)
+    double latency_us = 0.0; // estimated run time of the class's longest work item alone
     BandItem *d_items = nullptr;   // records + radix plans of the class's bands, longest first
     std::vector<int32_t> work;
 };
