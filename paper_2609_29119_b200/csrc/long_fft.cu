@@ -21,6 +21,8 @@
 // Weighted-bin scratch: P planes of Lp+1 bins per signal; band b writes plane b mod P, where P is the
 // largest number of bands covering one bin, so two bands of one plane never share a bin and the sum
 // over the bands covering bin k reads planes (lo + i) mod P, i < n, at index k: coalesced, no atomics.
+#include <algorithm>
+
 #include "engine.cuh"
 #include "internal.hpp"
 #include "static_fft.cuh"
@@ -546,7 +548,11 @@ static cudaError_t launch_long(const void *fn, dim3 grid, int threads, size_t sm
     return launch_kernel(fn, grid, dim3((unsigned)threads), args, smem, st);
 }
 
-static int threads_for(size_t butterflies) {
+// one thread per butterfly of the stage with the most butterflies (the smallest radix of the plan), up to 512
+static int threads_for(size_t elements, const FftPlan &fp) {
+    int rmin = 16;
+    for (int j = 0; j < fp.nstages; ++j) rmin = std::min(rmin, (int)fp.st[j].radix);
+    const size_t butterflies = elements / (size_t)std::max(rmin, 2);
     int t = 64;
     while (t < 512 && (size_t)t < butterflies) t *= 2;
     return t;
@@ -561,17 +567,17 @@ cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_str
     const LongFft &lf = p.lf;
     if (lf.A > 1) {
         dim3 grid((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
-        launch_long(cols_fwd_fn(p), grid, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), a, st);
+        launch_long(cols_fwd_fn(p), grid, threads_for((size_t)lf.A * lf.tw_cols, p.ffts[lf.fft_A]), cols_smem(p), a, st);
         note_launch(p, "rfft_cols_fwd", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         a.rows_magic = magic_of(2 * lf.tw_rows);
         dim3 grid2((unsigned)(lf.A / (2 * lf.tw_rows)), (unsigned)batch);
-        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows) / 8), rows_fwd_smem(p), a, st);
+        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B * (2 * lf.tw_rows), p.ffts[lf.fft_B]), rows_fwd_smem(p), a, st);
     } else {
         a.rows_magic = 0;
         dim3 grid2(1, (unsigned)batch);
-        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B / 8), rows_fwd_smem(p), a, st);
+        launch_long(rows_fwd_fn(p), grid2, threads_for((size_t)lf.B, p.ffts[lf.fft_B]), rows_fwd_smem(p), a, st);
     }
     note_launch(p, "rfft_rows_fwd", st);
     return cudaGetLastError();
@@ -588,17 +594,20 @@ cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, f
     if (lf.A > 1) {
         a.rows_magic = magic_of(2 * lf.tw_rows);
         dim3 grid((unsigned)(lf.A / (2 * lf.tw_rows)), (unsigned)batch);
-        launch_long(rows_inv_fn(p), grid, threads_for((size_t)lf.B * (2 * lf.tw_rows) / 8), rows_inv_smem(p), a, st);
+        // the overlap-add prologue is a latency chain per thread: with fewer CTAs than SMs it takes every thread it can get
+        const bool few = (long long)grid.x * grid.y < (long long)p.sm_count;
+        const int thr = few ? 512 : threads_for((size_t)lf.B * (2 * lf.tw_rows), p.ffts[lf.fft_B]);
+        launch_long(rows_inv_fn(p), grid, thr, rows_inv_smem(p), a, st);
         note_launch(p, "irfft_rows", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         dim3 grid2((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
-        launch_long(cols_inv_fn(p), grid2, threads_for((size_t)lf.A * lf.tw_cols / 8), cols_smem(p), a, st);
+        launch_long(cols_inv_fn(p), grid2, threads_for((size_t)lf.A * lf.tw_cols, p.ffts[lf.fft_A]), cols_smem(p), a, st);
         note_launch(p, "irfft_cols", st);
     } else {
         a.rows_magic = 0;
         dim3 grid(1, (unsigned)batch);
-        launch_long(rows_inv_fn(p), grid, threads_for((size_t)lf.B / 8), rows_inv_smem(p), a, st);
+        launch_long(rows_inv_fn(p), grid, threads_for((size_t)lf.B, p.ffts[lf.fft_B]), rows_inv_smem(p), a, st);
         note_launch(p, "irfft_rows", st);
     }
     return cudaGetLastError();
