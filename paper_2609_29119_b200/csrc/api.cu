@@ -339,7 +339,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
         br.fft = -1;
     }
     // ---- launch classes by band length
-    // class 0: one warp per item, 8 items per CTA; the others one CTA per item, sized so that several CTAs
+    // class 0: 8 lanes per item, 32 items per CTA; the others one CTA per item, sized so that several CTAs
     // share an SM (64 registers per thread) except for the longest bands, which fill its shared memory
     const int limits[kNumClasses] = {128, 1024, 4096, 13500, 1 << 30};
     {
@@ -348,7 +348,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
         for (int c = 0; c < kNumClasses; ++c) {
             p->cls[c].threads = threads[c];
             p->cls[c].min_blocks = minb[c];
-            p->cls[c].items_per_cta = c == 0 ? 8 : 1;
+            p->cls[c].multi_item = c == 0;
             p->cls[c].max_radix = c <= 1 ? 8 : (c == 2 ? 12 : 16);
         }
     }
@@ -403,7 +403,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
             const FftPlan &bf = p->ffts[p->bands[i].fft];
             const int64_t elems = bf.generic == 2 ? bf.blu_L + p->ffts[bf.blu_fft].tw_count
                                                   : (bf.generic ? 2 * M + bf.st[0].radix : M + 16 + bf.tw_count);
-            if (elems * p->cls[c].items_per_cta > smem_cap_elems) {
+            if (elems > smem_cap_elems) {   // the cap is per work item; the classes with several items per CTA are far below it
                 A2 = split_two_pass(M);
                 if (!A2) { delete p; return CQT_ERR_UNSUPPORTED; }
                 single = false;
@@ -436,6 +436,8 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
             g.smem_rows = std::max(g.smem_rows, two_pass_smem_rows(tb));
         }
     }
+    // a middle class whose longest band has at most one butterfly per thread at half the threads runs narrower CTAs
+    if (p->cls[2].n_bands && L.bands[(size_t)p->cls[2].work[0]].M <= 2304) { p->cls[2].threads = 128; p->cls[2].min_blocks = 8; }
     // estimates for the per-call assignment of classes to streams (band.cu): total work, and the time one CTA
     // needs for the longest item (microseconds per element by class, from measured kernel times)
     {
@@ -508,8 +510,12 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
     chk(cudaGetDeviceProperties(&prop, p->device));
     p->sm_count = prop.multiProcessorCount;
     p->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    // the helper streams carry the shorter classes: at the highest priority their CTAs are placed ahead of the
+    // long class on the caller's stream, whatever order the launches (or the nodes of a captured graph) arrive in
+    int prio_least = 0, prio_greatest = 0;
+    chk(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
     for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
-        chk(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
+        chk(cudaStreamCreateWithPriority(&p->aux[i], cudaStreamNonBlocking, prio_greatest));
         chk(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
     }
     chk(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));

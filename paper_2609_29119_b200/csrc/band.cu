@@ -22,12 +22,21 @@ static BandArgs make_args(const cqt_plan &p, const BandClass &c, const float *ta
     return a;
 }
 
-const void *band_analysis_kernel(const BandClass &c);    // band_analysis.cu
-const void *band_synthesis_kernel(const BandClass &c);   // band_synthesis.cu
+const void *band_analysis_kernel(const BandClass &c, int lanes);    // band_analysis.cu
+const void *band_synthesis_kernel(const BandClass &c, int lanes);   // band_synthesis.cu
 
 template <bool ANALYSIS>
-static const void *class_kernel(const BandClass &c) {
-    return ANALYSIS ? band_analysis_kernel(c) : band_synthesis_kernel(c);
+static const void *class_kernel(const BandClass &c, int lanes) {
+    return ANALYSIS ? band_analysis_kernel(c, lanes) : band_synthesis_kernel(c, lanes);
+}
+
+// Lanes per work item of the class of the shortest bands (0: the class gives every item a whole CTA).  A band of at
+// most 128 coefficients has at most 16 radix-8 butterflies per stage, so 8 lanes per item keep the lanes busy: fewer
+// warps for the same work, which leaves the SMs to the long-band classes running beside it.  A whole warp per item
+// has the shorter critical path, which is what counts in a call with few items (a single signal, one streaming hop).
+static int lanes_for(const cqt_plan &p, const BandClass &c, long long items) {
+    if (!c.multi_item) return 0;
+    return items >= 8ll * p.sm_count ? 8 : 32;
 }
 
 template <bool ANALYSIS>
@@ -35,10 +44,12 @@ static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, Ba
     const BandClass &c = p.cls[cls];
     if (c.n_bands == 0) return cudaSuccess;
     const long long items = (long long)c.n_bands * a.batch;
-    const size_t smem = (size_t)c.max_elems * c.items_per_cta * sizeof(float2);
-    const long long grid = (items + c.items_per_cta - 1) / c.items_per_cta;
+    const int lanes = lanes_for(p, c, items);
+    const int per_cta = lanes ? c.threads / lanes : 1;
+    const size_t smem = (size_t)c.max_elems * per_cta * sizeof(float2);
+    const long long grid = (items + per_cta - 1) / per_cta;
     void *args[] = {&a};
-    const void *fn = class_kernel<ANALYSIS>(c);
+    const void *fn = class_kernel<ANALYSIS>(c, lanes);
     if (!fn) return cudaErrorInvalidDeviceFunction;
     cudaError_t e = launch_kernel(fn, dim3((unsigned)grid), dim3(c.threads), args, smem, st);
     note_launch(p, name, st);
@@ -142,13 +153,16 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
 
 cudaError_t configure_band_kernels(const cqt_plan &p) {
     for (int i = 0; i < kNumClasses; ++i) {
-        const size_t s = (size_t)p.cls[i].max_elems * p.cls[i].items_per_cta * sizeof(float2);
         if (p.cls[i].n_bands == 0) continue;
-        if (!class_kernel<true>(p.cls[i])) return cudaErrorInvalidDeviceFunction;
-        cudaError_t e = allow_dynamic_smem(class_kernel<true>(p.cls[i]), s, p);
-        if (e != cudaSuccess) return e;
-        e = allow_dynamic_smem(class_kernel<false>(p.cls[i]), s, p);
-        if (e != cudaSuccess) return e;
+        for (int lanes : {0, 8, 32}) {
+            if ((lanes != 0) != p.cls[i].multi_item) continue;
+            const size_t s = (size_t)p.cls[i].max_elems * (lanes ? p.cls[i].threads / lanes : 1) * sizeof(float2);
+            if (!class_kernel<true>(p.cls[i], lanes)) return cudaErrorInvalidDeviceFunction;
+            cudaError_t e = allow_dynamic_smem(class_kernel<true>(p.cls[i], lanes), s, p);
+            if (e != cudaSuccess) return e;
+            e = allow_dynamic_smem(class_kernel<false>(p.cls[i], lanes), s, p);
+            if (e != cudaSuccess) return e;
+        }
     }
     return cudaSuccess;
 }

@@ -3,15 +3,15 @@
 
 namespace cqt {
 
-template <int THREADS, int MINB, bool WARP, int MAXR, bool GEN>
+template <int THREADS, int MINB, int LANES, int MAXR, bool GEN>
 __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(BandArgs a) {
     pdl_launch_dependents();
-    using G = Group<WARP>;
-    using Sync = typename std::conditional<WARP, WarpSync, BlockSync>::type;
+    using G = Group<LANES>;
+    using Sync = GroupSync<LANES>;
     const int item = G::item();
     if (item >= a.n_work * a.batch) return;   // whole group exits together
     const int tid = G::tid(), nthr = G::nthr();
-    __shared__ BandItem item_s[WARP ? 8 : 1];
+    __shared__ BandItem item_s[LANES ? THREADS / (LANES ? LANES : 1) : 1];
     BandItem &it = item_s[G::slot()];
     fetch_item<Sync>(a.items[item / a.batch], it, tid, nthr);   // records in launch order of the class
     const BandRec br = it.br;
@@ -80,9 +80,9 @@ __global__ void __launch_bounds__(THREADS, MINB) bands_from_spectrum_kernel(Band
     fft_fused<+1, Sync, false, true, false, true, false, false, MAXR>(t, fp, tws, load, store, tid, nthr);
 }
 
-const void *band_analysis_kernel(const BandClass &c) {
+const void *band_analysis_kernel(const BandClass &c, int lanes) {
 #define X(T, B, W, R)                                                                          \
-    if (c.threads == T && c.min_blocks == B && (c.items_per_cta > 1) == W && c.max_radix <= R)  \
+    if (c.threads == T && c.min_blocks == B && lanes == W && c.max_radix <= R)  \
         return c.has_generic ? (const void *)bands_from_spectrum_kernel<T, B, W, R, true> : (const void *)bands_from_spectrum_kernel<T, B, W, R, false>;
     CQT_KERNEL_TABLE(X)
 #undef X

@@ -36,13 +36,19 @@ struct BandArgs {
 };
 
 // THREADS / MINB: launch bounds of the class (64 registers per thread when THREADS * MINB = 1024 ... 2048)
-template <bool WARP>
+// LANES: 0 = the whole CTA works on one item; 32, 16, 8 = that many consecutive lanes per item (THREADS / LANES items
+// per CTA): the shortest bands have fewer butterflies per stage than a warp has lanes
+template <int LANES>
 struct Group {
-    __device__ static int tid() { return WARP ? (threadIdx.x & 31) : threadIdx.x; }
-    __device__ static int nthr() { return WARP ? 32 : blockDim.x; }
-    __device__ static int item() { return WARP ? blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5) : blockIdx.x; }
-    __device__ static int slot() { return WARP ? (threadIdx.x >> 5) : 0; }
+    __device__ static int tid() { return LANES ? (int)(threadIdx.x & (LANES - 1)) : (int)threadIdx.x; }
+    __device__ static int nthr() { return LANES ? LANES : (int)blockDim.x; }
+    __device__ static int per_cta() { return LANES ? (int)blockDim.x / (LANES ? LANES : 1) : 1; }
+    __device__ static int slot() { return LANES ? (int)threadIdx.x / (LANES ? LANES : 1) : 0; }
+    __device__ static int item() { return LANES ? (int)blockIdx.x * per_cta() + slot() : (int)blockIdx.x; }
 };
+template <int LANES>
+using GroupSync = typename std::conditional<LANES == 0, BlockSync,
+                                            typename std::conditional<LANES == 32, WarpSync, LaneGroupSync<(LANES ? LANES : 1)>>::type>::type;
 
 extern __shared__ float2 smem_band[];
 
@@ -92,10 +98,10 @@ __device__ __forceinline__ void chirp_z_transform(float2 *buf, const FftPlan &fp
     }
 }
 
-// Kernel instantiations: (threads per CTA, CTAs per SM the registers must allow, one warp per item, largest radix
+// Kernel instantiations: (threads per CTA, CTAs per SM the registers must allow, lanes per item or 0 for the whole CTA, largest radix
 // compiled in), each with and without the prime-factor paths (GEN): code a class never runs is left out, which also
 // frees registers in the paths it does run.
 #define CQT_KERNEL_TABLE(X) \
-    X(256, 4, true, 8) X(64, 16, false, 8) X(256, 4, false, 12) X(512, 2, false, 16) X(1024, 1, false, 16)
+    X(256, 4, 8, 8) X(256, 4, 32, 8) X(64, 16, 0, 8) X(128, 8, 0, 12) X(256, 4, 0, 12) X(512, 2, 0, 16) X(1024, 1, 0, 16)
 
 }  // namespace cqt

@@ -26,6 +26,14 @@ struct BlockSync {
 struct WarpSync {
     static __device__ __forceinline__ void sync() { __syncwarp(); }
 };
+// LANES consecutive lanes of a warp (a power of two below 32) working on one item: the groups of a warp may be in
+// different places of the code (items with different radix plans), so each synchronises with its own lane mask
+template <int LANES>
+struct LaneGroupSync {
+    static __device__ __forceinline__ void sync() {
+        __syncwarp(((1u << LANES) - 1u) << ((threadIdx.x & 31u) & ~(unsigned)(LANES - 1)));
+    }
+};
 
 __device__ __forceinline__ float2 cmul(float2 a, float2 b) {
     return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
