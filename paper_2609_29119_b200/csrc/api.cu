@@ -348,7 +348,8 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
         for (int c = 0; c < kNumClasses; ++c) {
             p->cls[c].threads = threads[c];
             p->cls[c].min_blocks = minb[c];
-            p->cls[c].multi_item = c == 0;
+            p->cls[c].lanes_few = c == 0 ? 32 : 0;
+            p->cls[c].lanes_many = c == 0 ? 8 : 0;
             p->cls[c].max_radix = c <= 1 ? 8 : (c == 2 ? 12 : 16);
         }
     }

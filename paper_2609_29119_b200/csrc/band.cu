@@ -35,8 +35,7 @@ static const void *class_kernel(const BandClass &c, int lanes) {
 // warps for the same work, which leaves the SMs to the long-band classes running beside it.  A whole warp per item
 // has the shorter critical path, which is what counts in a call with few items (a single signal, one streaming hop).
 static int lanes_for(const cqt_plan &p, const BandClass &c, long long items) {
-    if (!c.multi_item) return 0;
-    return items >= 8ll * p.sm_count ? 8 : 32;
+    return items >= 8ll * p.sm_count ? c.lanes_many : c.lanes_few;
 }
 
 template <bool ANALYSIS>
@@ -154,8 +153,7 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
 cudaError_t configure_band_kernels(const cqt_plan &p) {
     for (int i = 0; i < kNumClasses; ++i) {
         if (p.cls[i].n_bands == 0) continue;
-        for (int lanes : {0, 8, 32}) {
-            if ((lanes != 0) != p.cls[i].multi_item) continue;
+        for (int lanes : {p.cls[i].lanes_few, p.cls[i].lanes_many}) {
             const size_t s = (size_t)p.cls[i].max_elems * (lanes ? p.cls[i].threads / lanes : 1) * sizeof(float2);
             if (!class_kernel<true>(p.cls[i], lanes)) return cudaErrorInvalidDeviceFunction;
             cudaError_t e = allow_dynamic_smem(class_kernel<true>(p.cls[i], lanes), s, p);

@@ -16,7 +16,8 @@ constexpr int kNumClasses = 5;
 struct BandClass {
     int threads = 0;         // threads per CTA
     int min_blocks = 1;      // CTAs per SM the kernel instantiation is compiled for (register budget)
-    bool multi_item = false; // several (band, signal) items per CTA, 8 or 32 lanes each (chosen per call)
+    int lanes_few = 0, lanes_many = 0;   // > 0: several (band, signal) items per CTA, that many lanes each, in a call
+                                         // with few / many items; 0: one item per CTA
     int max_radix = 16;      // largest butterfly radix in the class's plans
     bool has_generic = false; // some band of the class has a prime factor above 5 (direct-sum stage or chirp-z)
     int max_elems = 0;       // shared-memory elements (float2) per item
