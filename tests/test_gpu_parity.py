@@ -26,6 +26,12 @@ CASES = [
                    m_policy=wl.M_SMOOTH, channels=3),
     small_workload("n4096_ragged", N=4096, valid_len=3001, fs=22050.0, fmin=200.0, fmax=11025.0, bins_per_octave=12,
                    m_policy=wl.M_MULT4, channels=3),
+    # enough (band, signal) items for the lane-group kernels of the shortest bands (8 lanes per item), on lengths
+    # with prime factors above 5 (direct-sum stage) and on 5-smooth ones
+    small_workload("n4096_b48_mult4_48ch", N=4096, valid_len=3900, fs=22050.0, fmin=200.0, fmax=11025.0,
+                   bins_per_octave=48, m_policy=wl.M_MULT4, channels=48),
+    small_workload("n4096_b48_smooth_40ch", N=4096, valid_len=4096, fs=22050.0, fmin=200.0, fmax=11025.0,
+                   bins_per_octave=48, m_policy=wl.M_SMOOTH, window=wl.WIN_BLACKMAN_HARRIS, channels=40),
     small_workload("n16384_mult4", N=1 << 14, valid_len=1 << 14, fs=44100.0, fmin=32.70, fmax=22050.0,
                    bins_per_octave=12, m_policy=wl.M_MULT4, channels=2),
     small_workload("slice_2e15", N=1 << 15, valid_len=1 << 15, fs=44100.0, fmin=32.70, fmax=22050.0,
@@ -125,6 +131,22 @@ def test_bitwise_reproducible(case):
     x1 = plan.synthesise(c1, valid_len=w.valid_len)
     x2 = plan.synthesise(c1, valid_len=w.valid_len)
     assert torch.equal(x1, x2)
+
+
+def test_results_do_not_depend_on_the_batch_size():
+    """A signal's coefficients and reconstruction are bitwise the same whether it is transformed alone or in a
+    large batch (the launch shapes differ: lanes per item of the shortest bands, threads of the long FFT)."""
+    w = small_workload("n4096_b48_mult4_64ch", N=4096, valid_len=4001, fs=22050.0, fmin=200.0, fmax=11025.0,
+                       bins_per_octave=48, m_policy=wl.M_MULT4, channels=64)
+    plan = library_plan(w)
+    xd = _dev(wl.make_signal(w))
+    c_all = plan.analyse(xd, valid_len=w.valid_len)
+    x_all = plan.synthesise(c_all, valid_len=w.valid_len)
+    for rows in (slice(0, 1), slice(61, 64)):
+        c = plan.analyse(xd[rows].contiguous(), valid_len=w.valid_len)
+        assert torch.equal(torch.view_as_real(c), torch.view_as_real(c_all[rows]))
+        assert torch.equal(plan.synthesise(c, valid_len=w.valid_len), x_all[rows])
+    plan.close()
 
 
 def test_row_stride_and_padding_are_respected():
