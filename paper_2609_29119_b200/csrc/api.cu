@@ -183,7 +183,7 @@ void free_device(cqt_plan *p) {
     for (auto &c : p->cls) cudaFree(c.d_items);
     for (auto &g : p->two_pass) cudaFree(g.d_recs);
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < cqt_plan::kHelpers; ++i) {
         if (p->aux[i]) cudaStreamDestroy(p->aux[i]);
         if (p->ev_join[i]) cudaEventDestroy(p->ev_join[i]);
     }
@@ -515,7 +515,7 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
     // long class on the caller's stream, whatever order the launches (or the nodes of a captured graph) arrive in
     int prio_least = 0, prio_greatest = 0;
     chk(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
-    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    for (int i = 0; i < cqt_plan::kHelpers && e == cudaSuccess; ++i) {
         chk(cudaStreamCreateWithPriority(&p->aux[i], cudaStreamNonBlocking, prio_greatest));
         chk(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
     }

@@ -56,7 +56,8 @@ static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, Ba
 }
 
 // The classes of one call are independent (disjoint outputs), and most of them alone leave SMs idle, so they run
-// side by side on the caller's stream and two helper streams: fork after the caller's stream, join back into it.
+// side by side on the caller's stream and the plan's helper streams (one stream per class when all five classes
+// have bands): fork after the caller's stream, join back into it.
 // Per call, each class's run time is estimated as the larger of the time of its longest work item and its work
 // at this batch size over the machine's throughput; the classes go, longest first, to the stream with the least
 // time so far (the longest one therefore stays on the caller's stream).  With event timing on, everything stays
@@ -64,14 +65,14 @@ static cudaError_t launch_class(const cqt_plan &p, int cls, const char *name, Ba
 struct ForkJoin {
     const cqt_plan &p;
     cudaStream_t st;
-    bool used[2] = {false, false};
+    bool used[cqt_plan::kHelpers] = {};
     bool serial;
     int slot[kNumClasses] = {0, 0, 0, 0, 0};
     ForkJoin(const cqt_plan &plan, cudaStream_t s, int64_t batch)
-        : p(plan), st(s), serial(plan.timing || !plan.aux[0] || !plan.aux[1]) {
+        : p(plan), st(s), serial(plan.timing || !plan.aux[cqt_plan::kHelpers - 1]) {
         if (serial) return;
         constexpr double kElementStagesPerUs = 6.7e5;   // the 4096 < M <= 13,500 class at 32 signals
-        double est[kNumClasses], load[3] = {0.0, 0.0, 0.0};
+        double est[kNumClasses], load[cqt_plan::kHelpers + 1] = {};
         int order[kNumClasses];
         for (int c = 0; c < kNumClasses; ++c) {
             order[c] = c;
@@ -82,7 +83,7 @@ struct ForkJoin {
             const int c = order[i];
             if (!p.cls[c].n_bands) continue;
             int best = 0;
-            for (int j = 1; j < 3; ++j)
+            for (int j = 1; j <= cqt_plan::kHelpers; ++j)
                 if (load[j] < load[best]) best = j;
             slot[c] = best;
             load[best] += est[c];
@@ -96,7 +97,7 @@ struct ForkJoin {
         return p.aux[i];
     }
     void join() {
-        for (int i = 0; i < 2; ++i)
+        for (int i = 0; i < cqt_plan::kHelpers; ++i)
             if (used[i]) { cudaEventRecord(p.ev_join[i], p.aux[i]); cudaStreamWaitEvent(st, p.ev_join[i], 0); }
     }
 };

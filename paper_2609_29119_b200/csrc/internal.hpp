@@ -82,8 +82,9 @@ struct cqt_plan {
     int max_smem_optin = 0;
     int sm_count = 0;
     // helper streams on which the short-band classes run beside the long-band classes of the same call
-    cudaStream_t aux[2] = {nullptr, nullptr};
-    cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr};
+    static constexpr int kHelpers = 4;
+    cudaStream_t aux[kHelpers] = {};
+    cudaEvent_t ev_fork = nullptr, ev_join[kHelpers] = {};
     // launch counter and optional per-kernel event timing (benchmark aid; not thread safe)
     mutable int64_t launches = 0;
     mutable bool timing = false;
