@@ -24,7 +24,7 @@
  *             256-byte aligned; contents are undefined after a call.  Calls that run
  *             concurrently on different streams need different workspaces.
  *   stream    a cudaStream_t passed as void*; all transform calls are asynchronous
- *             on it and never synchronise the device.  A plan owns four helper streams
+ *             on it and never synchronise the device.  A plan owns five helper streams
  *             that fork from and join the caller's stream inside every call (the calls
  *             can be captured in a CUDA graph).
  *   threads   calls on ONE plan (or one cqt_slicq) must come from one host thread at a

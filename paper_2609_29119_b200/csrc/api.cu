@@ -668,8 +668,7 @@ cqt_status run_analysis_form(const cqt_plan *p, const float *table, const float 
     cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
     if (s != CQT_OK) return s;
     cudaError_t e = launch_rfft_forward(*p, x, x_stride, batch, valid_len, k.T, k.second, k.st);
-    if (e == cudaSuccess) e = launch_two_pass_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), k.huge, batch, k.st);
-    if (e == cudaSuccess) e = launch_bands_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), batch, k.st);
+    if (e == cudaSuccess) e = launch_bands_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), k.huge, batch, k.st);
     return end_call(k, e);
 }
 
@@ -678,8 +677,7 @@ cqt_status run_synthesis_form(const cqt_plan *p, const float *table, bool fold, 
     Call k;
     cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
     if (s != CQT_OK) return s;
-    cudaError_t e = launch_two_pass_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, k.huge, batch, k.st);
-    if (e == cudaSuccess) e = launch_bands_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, batch, k.st);
+    cudaError_t e = launch_bands_to_spectrum(*p, table, fold, reinterpret_cast<const float2 *>(c), k.second, k.huge, batch, k.st);
     if (e == cudaSuccess) e = launch_rfft_inverse(*p, k.second, k.T, x, x_stride, batch, valid_len, k.st);
     return end_call(k, e);
 }

@@ -72,7 +72,7 @@ struct ForkJoin {
         : p(plan), st(s), serial(plan.timing || !plan.aux[cqt_plan::kHelpers - 1]) {
         if (serial) return;
         constexpr double kElementStagesPerUs = 6.7e5;   // the 4096 < M <= 13,500 class at 32 signals
-        double est[kNumClasses], load[cqt_plan::kHelpers + 1] = {};
+        double est[kNumClasses], load[cqt_plan::kHelpers] = {};   // the last helper is kept for the two-pass bands
         int order[kNumClasses];
         for (int c = 0; c < kNumClasses; ++c) {
             order[c] = c;
@@ -83,7 +83,7 @@ struct ForkJoin {
             const int c = order[i];
             if (!p.cls[c].n_bands) continue;
             int best = 0;
-            for (int j = 1; j <= cqt_plan::kHelpers; ++j)
+            for (int j = 1; j < cqt_plan::kHelpers; ++j)
                 if (load[j] < load[best]) best = j;
             slot[c] = best;
             load[best] += est[c];
@@ -96,6 +96,12 @@ struct ForkJoin {
         if (!used[i]) { cudaStreamWaitEvent(p.aux[i], p.ev_fork, 0); used[i] = true; }
         return p.aux[i];
     }
+    cudaStream_t two_pass_stream() {
+        if (serial) return st;
+        const int i = cqt_plan::kHelpers - 1;
+        if (!used[i]) { cudaStreamWaitEvent(p.aux[i], p.ev_fork, 0); used[i] = true; }
+        return p.aux[i];
+    }
     void join() {
         for (int i = 0; i < cqt_plan::kHelpers; ++i)
             if (used[i]) { cudaEventRecord(p.ev_join[i], p.aux[i]); cudaStreamWaitEvent(st, p.ev_join[i], 0); }
@@ -103,8 +109,12 @@ struct ForkJoin {
 };
 
 cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
-                                       int64_t batch, cudaStream_t st) {
+                                       float2 *scratch, int64_t batch, cudaStream_t st) {
     ForkJoin fj(p, st, batch);
+    if (!p.two_pass[0].bands.empty() || !p.two_pass[1].bands.empty()) {
+        cudaError_t e = launch_two_pass_from_spectrum(p, table, X, c, scratch, batch, fj.two_pass_stream());
+        if (e != cudaSuccess) { fj.join(); return e; }
+    }
     static const char *names[kNumClasses] = {"bands_from_spectrum/class0", "bands_from_spectrum/class1",
                                               "bands_from_spectrum/class2", "bands_from_spectrum/class3",
                                               "bands_from_spectrum/class4"};
@@ -128,7 +138,7 @@ __global__ void __launch_bounds__(128) zero_fill_kernel(float2 *Y, long long y_p
 }
 
 cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool fold_sidebands, const float2 *c,
-                                     float2 *Y, int64_t batch, cudaStream_t st) {
+                                     float2 *Y, float2 *scratch, int64_t batch, cudaStream_t st) {
     if (p.n_zero_seg > 0) {
         zero_fill_kernel<<<dim3((unsigned)p.n_zero_seg, (unsigned)batch), 128, 0, st>>>(Y, p.y_pitch, p.d.zero_seg);
         note_launch(p, "zero_fill", st);
@@ -136,6 +146,10 @@ cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool
         if (e != cudaSuccess) return e;
     }
     ForkJoin fj(p, st, batch);
+    if (!p.two_pass[0].bands.empty() || !p.two_pass[1].bands.empty()) {
+        cudaError_t e = launch_two_pass_to_spectrum(p, table, fold_sidebands, c, Y, scratch, batch, fj.two_pass_stream());
+        if (e != cudaSuccess) { fj.join(); return e; }
+    }
     static const char *names[kNumClasses] = {"bands_to_spectrum/class0", "bands_to_spectrum/class1",
                                               "bands_to_spectrum/class2", "bands_to_spectrum/class3",
                                               "bands_to_spectrum/class4"};

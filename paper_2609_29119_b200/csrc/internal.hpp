@@ -82,7 +82,7 @@ struct cqt_plan {
     int max_smem_optin = 0;
     int sm_count = 0;
     // helper streams on which the short-band classes run beside the long-band classes of the same call
-    static constexpr int kHelpers = 4;
+    static constexpr int kHelpers = 5;   // one per band class beside the caller's stream, one for the two-pass bands
     cudaStream_t aux[kHelpers] = {};
     cudaEvent_t ev_fork = nullptr, ev_join[kHelpers] = {};
     // launch counter and optional per-kernel event timing (benchmark aid; not thread safe)
@@ -152,10 +152,12 @@ inline cudaError_t launch_kernel_args(void (*kernel)(KArgs...), dim3 grid, dim3 
 }
 
 // band.cu
+// every band of the plan: the single-CTA classes and, beside them on a stream of their own, the two-pass bands
+// (scratch: their rows in the workspace)
 cudaError_t launch_bands_from_spectrum(const cqt_plan &p, const float *table, const float2 *X, float2 *c,
-                                       int64_t batch, cudaStream_t st);
+                                       float2 *scratch, int64_t batch, cudaStream_t st);
 cudaError_t launch_bands_to_spectrum(const cqt_plan &p, const float *table, bool fold_sidebands, const float2 *c,
-                                     float2 *Y, int64_t batch, cudaStream_t st);
+                                     float2 *Y, float2 *scratch, int64_t batch, cudaStream_t st);
 cudaError_t configure_band_kernels(const cqt_plan &p);
 
 // band_two_pass.cu
