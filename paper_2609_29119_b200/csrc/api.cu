@@ -430,11 +430,13 @@ static cqt_status finish_plan(cqt_plan *p, int64_t N, int device, const cqt_plan
             p->two_pass_pitch += (M + 7) / 8 * 8;
             TwoPassGroup &g = p->two_pass[(tb.A <= 256 && tb.B <= 256) ? 0 : 1];
             g.bands.push_back(tb);
-            const int tw_tile = two_pass_tile();
-            g.max_tiles_cols = std::max(g.max_tiles_cols, (tb.B + tw_tile - 1) / tw_tile);
-            g.max_tiles_rows = std::max(g.max_tiles_rows, (tb.A + tw_tile - 1) / tw_tile);
-            g.smem_cols = std::max(g.smem_cols, two_pass_smem_cols(tb));
-            g.smem_rows = std::max(g.smem_rows, two_pass_smem_rows(tb));
+            for (int wi = 0; wi < 3; ++wi) {
+                const int tw_tile = kTwoPassWidths[wi];
+                g.max_tiles_cols[wi] = std::max(g.max_tiles_cols[wi], (tb.B + tw_tile - 1) / tw_tile);
+                g.max_tiles_rows[wi] = std::max(g.max_tiles_rows[wi], (tb.A + tw_tile - 1) / tw_tile);
+                g.smem_cols[wi] = std::max(g.smem_cols[wi], two_pass_smem_cols(tb, tw_tile));
+                g.smem_rows[wi] = std::max(g.smem_rows[wi], two_pass_smem_rows(tb, tw_tile));
+            }
         }
     }
     // a middle class whose longest band has at most one butterfly per thread at half the threads runs narrower CTAs

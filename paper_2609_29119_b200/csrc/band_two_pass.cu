@@ -18,7 +18,6 @@ namespace cqt {
 
 extern __shared__ float2 smem_tp[];
 
-constexpr int kTW = 16;   // columns (pass 1) / rows (pass 2) per CTA
 
 struct TwoPassArgs {
     const TwoPassRec *recs;
@@ -62,26 +61,26 @@ __device__ __forceinline__ void copy_table(float2 *dst, const float2 *__restrict
     for (int i = tid; i < n; i += nthr) dst[i] = __ldg(src + i);
 }
 
-// pass 1: kTW adjacent columns (second index), A-point transform over the first index, inter-pass twiddle
-template <int THREADS, int MINB, bool ANALYSIS>
+// pass 1: TW adjacent columns (second index), A-point transform over the first index, inter-pass twiddle
+template <int THREADS, int MINB, bool ANALYSIS, int TW>
 __global__ void __launch_bounds__(THREADS, MINB) band2p_cols_kernel(TwoPassArgs a) {
     pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const TwoPassRec rec = a.recs[blockIdx.y / a.groups];
     const int ch0 = (blockIdx.y % a.groups) * a.ch_per_cta, ch1 = min(a.batch, ch0 + a.ch_per_cta);
-    const int c0 = blockIdx.x * kTW;
+    const int c0 = blockIdx.x * TW;
     if (c0 >= rec.B) return;
-    const int ncols = min(kTW, rec.B - c0);
+    const int ncols = min(TW, rec.B - c0);
     const BandRec br = a.bands[rec.band];
     const FftPlan &fp = a.ffts[rec.fft_A];
     float2 *buf = smem_tp;
-    float2 *twf = buf + (size_t)rec.A * kTW;
+    float2 *twf = buf + (size_t)rec.A * TW;
     float2 *wm = twf + rec.A;
     copy_table(twf, a.tw + fp.tw_full_off, rec.A, tid, nthr);
     copy_table(wm, a.tw + rec.tw_m, rec.n_m, tid, nthr);
     const float *tab = a.table + br.tab_off;
     const bool fold = !ANALYSIS && a.fold && br.side != 0;
-    const Tile t{buf, kTW, kTW, 1u << 28, rec.A * kTW, a.dbg};
+    const Tile t{buf, TW, TW, 0x80000000u / (TW / 2), rec.A * TW, a.dbg};
     pdl_wait();   // tables and records belong to the plan; the loop touches the predecessor's output
     for (int ch = ch0; ch < ch1; ++ch) {
     const float2 *X = ANALYSIS ? a.spec + (long long)ch * a.spec_pitch : nullptr;
@@ -106,23 +105,23 @@ __global__ void __launch_bounds__(THREADS, MINB) band2p_cols_kernel(TwoPassArgs 
     }
 }
 
-// pass 2: kTW adjacent rows (first output index), B-point transform over the second index
-template <int THREADS, int MINB, bool ANALYSIS>
+// pass 2: TW adjacent rows (first output index), B-point transform over the second index
+template <int THREADS, int MINB, bool ANALYSIS, int TW>
 __global__ void __launch_bounds__(THREADS, MINB) band2p_rows_kernel(TwoPassArgs a) {
     pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const TwoPassRec rec = a.recs[blockIdx.y / a.groups];
     const int ch0 = (blockIdx.y % a.groups) * a.ch_per_cta, ch1 = min(a.batch, ch0 + a.ch_per_cta);
-    const int r0 = blockIdx.x * kTW;
+    const int r0 = blockIdx.x * TW;
     if (r0 >= rec.A) return;
-    const int nrows = min(kTW, rec.A - r0);
+    const int nrows = min(TW, rec.A - r0);
     const BandRec br = a.bands[rec.band];
     const FftPlan &fp = a.ffts[rec.fft_B];
     float2 *buf = smem_tp;
-    constexpr int pitch = kTW + 1;
+    constexpr int pitch = TW + 1;
     float2 *twf = buf + (size_t)rec.B * pitch;
     copy_table(twf, a.tw + fp.tw_full_off, rec.B, tid, nthr);
-    const Tile t{buf, pitch, kTW, 1u << 28, rec.B * pitch, a.dbg};
+    const Tile t{buf, pitch, TW, 0x80000000u / (TW / 2), rec.B * pitch, a.dbg};
     pdl_wait();   // tables and records belong to the plan; the loop touches the predecessor's output
     for (int ch = ch0; ch < ch1; ++ch) {
     const float2 *T = a.scratch + (long long)ch * a.scratch_pitch + rec.scratch_off;
@@ -160,16 +159,29 @@ __global__ void __launch_bounds__(THREADS, MINB) band2p_rows_kernel(TwoPassArgs 
     }
 }
 
-// group 0: both factors <= 256 (small tiles, 128 threads, many CTAs per SM); group 1: the rest
+// group 0: both factors <= 256 (small tiles, 128 threads at the full width, many CTAs per SM); group 1: the rest.
+// wi: index into kTwoPassWidths
 template <bool ANALYSIS>
-static const void *cols_kernel(int g) {
-    if (g == 1) return (const void *)band2p_cols_kernel<512, 2, ANALYSIS>;
-    return (const void *)band2p_cols_kernel<128, 8, ANALYSIS>;
+static const void *cols_kernel(int g, int wi) {
+    if (g == 1) {
+        if (wi == 0) return (const void *)band2p_cols_kernel<512, 2, ANALYSIS, 16>;
+        if (wi == 1) return (const void *)band2p_cols_kernel<512, 2, ANALYSIS, 8>;
+        return (const void *)band2p_cols_kernel<512, 2, ANALYSIS, 4>;
+    }
+    if (wi == 0) return (const void *)band2p_cols_kernel<128, 8, ANALYSIS, 16>;
+    if (wi == 1) return (const void *)band2p_cols_kernel<128, 8, ANALYSIS, 8>;
+    return (const void *)band2p_cols_kernel<128, 8, ANALYSIS, 4>;
 }
 template <bool ANALYSIS>
-static const void *rows_kernel(int g) {
-    if (g == 1) return (const void *)band2p_rows_kernel<512, 2, ANALYSIS>;
-    return (const void *)band2p_rows_kernel<128, 8, ANALYSIS>;
+static const void *rows_kernel(int g, int wi) {
+    if (g == 1) {
+        if (wi == 0) return (const void *)band2p_rows_kernel<512, 2, ANALYSIS, 16>;
+        if (wi == 1) return (const void *)band2p_rows_kernel<512, 2, ANALYSIS, 8>;
+        return (const void *)band2p_rows_kernel<512, 2, ANALYSIS, 4>;
+    }
+    if (wi == 0) return (const void *)band2p_rows_kernel<128, 8, ANALYSIS, 16>;
+    if (wi == 1) return (const void *)band2p_rows_kernel<128, 8, ANALYSIS, 8>;
+    return (const void *)band2p_rows_kernel<128, 8, ANALYSIS, 4>;
 }
 
 template <bool ANALYSIS>
@@ -191,21 +203,27 @@ static cudaError_t run_group(const cqt_plan &p, int g, const float *table, bool 
     a.Y = Y; a.y_pitch = p.y_pitch;
     a.scratch = scratch; a.scratch_pitch = p.two_pass_pitch;
     a.dbg = p.d.dbg;
+    // tile width: the widest whose grid still has a CTA for every SM (a single long signal has one huge band and a
+    // batch of one: 16-wide tiles would leave two thirds of the SMs without work), else the narrowest
+    int wi = 0;
+    while (wi < 2 && (long long)std::min(grp.max_tiles_cols[wi], grp.max_tiles_rows[wi]) * (long long)grp.bands.size() * batch < p.sm_count) ++wi;
+    // narrow tiles mean few CTAs: each keeps the full thread count, so that a thread has one or two butterflies per
+    // stage and the chain of dependent instructions per warp stays short
     const int threads = g == 0 ? 128 : 512;
     // signals per CTA: as many as keep at least ~6 CTAs per resident slot
     const long long slots = (long long)p.sm_count * (g == 0 ? 8 : 2);
-    const long long tiles = (long long)std::min(grp.max_tiles_cols, grp.max_tiles_rows) * (long long)grp.bands.size();
+    const long long tiles = (long long)std::min(grp.max_tiles_cols[wi], grp.max_tiles_rows[wi]) * (long long)grp.bands.size();
     int cpc = 1;
     while (cpc < 8 && tiles * ((batch + 2 * cpc - 1) / (2 * cpc)) >= 6 * slots) cpc *= 2;
     a.ch_per_cta = cpc;
     a.groups = (int)((batch + cpc - 1) / cpc);
     void *args[] = {&a};
-    dim3 g1((unsigned)grp.max_tiles_cols, (unsigned)(grp.bands.size() * a.groups));
-    cudaError_t e = launch_kernel(cols_kernel<ANALYSIS>(g), g1, dim3(threads), args, grp.smem_cols, st);
+    dim3 g1((unsigned)grp.max_tiles_cols[wi], (unsigned)(grp.bands.size() * a.groups));
+    cudaError_t e = launch_kernel(cols_kernel<ANALYSIS>(g, wi), g1, dim3(threads), args, grp.smem_cols[wi], st);
     note_launch(p, ANALYSIS ? (g ? "band2p_cols/analysis/large" : "band2p_cols/analysis") : (g ? "band2p_cols/synthesis/large" : "band2p_cols/synthesis"), st);
     if (e != cudaSuccess) return e;
-    dim3 g2((unsigned)grp.max_tiles_rows, (unsigned)(grp.bands.size() * a.groups));
-    e = launch_kernel(rows_kernel<ANALYSIS>(g), g2, dim3(threads), args, grp.smem_rows, st);
+    dim3 g2((unsigned)grp.max_tiles_rows[wi], (unsigned)(grp.bands.size() * a.groups));
+    e = launch_kernel(rows_kernel<ANALYSIS>(g, wi), g2, dim3(threads), args, grp.smem_rows[wi], st);
     note_launch(p, ANALYSIS ? (g ? "band2p_rows/analysis/large" : "band2p_rows/analysis") : (g ? "band2p_rows/synthesis/large" : "band2p_rows/synthesis"), st);
     return e;
 }
@@ -228,9 +246,8 @@ cudaError_t launch_two_pass_to_spectrum(const cqt_plan &p, const float *table, b
     return cudaSuccess;
 }
 
-size_t two_pass_smem_cols(const TwoPassBand &b) { return ((size_t)b.A * kTW + b.A + b.n_m) * sizeof(float2); }
-size_t two_pass_smem_rows(const TwoPassBand &b) { return ((size_t)b.B * (kTW + 1) + b.B) * sizeof(float2); }
-int two_pass_tile() { return kTW; }
+size_t two_pass_smem_cols(const TwoPassBand &b, int width) { return ((size_t)b.A * width + b.A + b.n_m) * sizeof(float2); }
+size_t two_pass_smem_rows(const TwoPassBand &b, int width) { return ((size_t)b.B * (width + 1) + b.B) * sizeof(float2); }
 
 cudaError_t configure_two_pass_kernels(const cqt_plan &p) {
     cudaError_t e = cudaSuccess;
@@ -239,10 +256,12 @@ cudaError_t configure_two_pass_kernels(const cqt_plan &p) {
     };
     for (int g = 0; g < 2; ++g) {
         if (p.two_pass[g].bands.empty()) continue;
-        set(cols_kernel<true>(g), p.two_pass[g].smem_cols);
-        set(cols_kernel<false>(g), p.two_pass[g].smem_cols);
-        set(rows_kernel<true>(g), p.two_pass[g].smem_rows);
-        set(rows_kernel<false>(g), p.two_pass[g].smem_rows);
+        for (int wi = 0; wi < 3; ++wi) {
+            set(cols_kernel<true>(g, wi), p.two_pass[g].smem_cols[wi]);
+            set(cols_kernel<false>(g, wi), p.two_pass[g].smem_cols[wi]);
+            set(rows_kernel<true>(g, wi), p.two_pass[g].smem_rows[wi]);
+            set(rows_kernel<false>(g, wi), p.two_pass[g].smem_rows[wi]);
+        }
     }
     return e;
 }

@@ -44,8 +44,9 @@ using TwoPassBand = TwoPassRec;
 struct TwoPassGroup {
     std::vector<TwoPassBand> bands;
     TwoPassRec *d_recs = nullptr;
-    int max_tiles_cols = 0, max_tiles_rows = 0;
-    size_t smem_cols = 0, smem_rows = 0;
+    // per tile width (kTwoPassWidths): CTAs along the tiled index and shared memory of the two passes
+    int max_tiles_cols[3] = {0, 0, 0}, max_tiles_rows[3] = {0, 0, 0};
+    size_t smem_cols[3] = {0, 0, 0}, smem_rows[3] = {0, 0, 0};
 };
 
 struct DevicePlan {
@@ -166,8 +167,9 @@ cudaError_t launch_two_pass_from_spectrum(const cqt_plan &p, const float *table,
 cudaError_t launch_two_pass_to_spectrum(const cqt_plan &p, const float *table, bool fold, const float2 *c, float2 *Y,
                                         float2 *scratch, int64_t batch, cudaStream_t st);
 cudaError_t configure_two_pass_kernels(const cqt_plan &p);
-size_t two_pass_smem_cols(const TwoPassBand &b);
-size_t two_pass_smem_rows(const TwoPassBand &b);
-int two_pass_tile();
+// tile widths (columns of pass 1 / rows of pass 2 per CTA) the kernels are compiled for, widest first
+constexpr int kTwoPassWidths[3] = {16, 8, 4};
+size_t two_pass_smem_cols(const TwoPassBand &b, int width);
+size_t two_pass_smem_rows(const TwoPassBand &b, int width);
 
 }  // namespace cqt

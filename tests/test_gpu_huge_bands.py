@@ -16,11 +16,13 @@ def _dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def test_two_pass_bands_match_oracle_with_a_lowered_cap():
+@pytest.mark.parametrize("channels", [1, 4, 12])
+def test_two_pass_bands_match_oracle_with_a_lowered_cap(channels):
     """With the per-CTA cap lowered, every band above 600 coefficients takes the two-pass kernels; all four
-    transforms are then compared with the oracle in full."""
+    transforms are then compared with the oracle in full.  The batch sizes make the launcher pick each of its
+    three tile widths (the fewer work items, the narrower the tiles)."""
     w = small_workload("forced_two_pass", N=1 << 14, valid_len=15000, fs=44100.0, fmin=32.70, fmax=22050.0,
-                       bins_per_octave=12, m_policy=wl.M_SMOOTH, channels=2, kind="noise_sines")
+                       bins_per_octave=12, m_policy=wl.M_SMOOTH, channels=channels, kind="noise_sines")
     plan = library_plan(w, max_cta_elems=600)
     lay = oracle_layout(w)
     assert max(b.M for b in lay.bands) > 600
