@@ -665,11 +665,12 @@ cqt_status end_call(const Call &c, cudaError_t e) {
 }
 
 cqt_status run_analysis_form(const cqt_plan *p, const float *table, const float *x, int64_t x_stride, int64_t batch,
-                             int64_t valid_len, cqt_c64 *c, void *ws, size_t ws_bytes, void *stream) {
+                             int64_t valid_len, cqt_c64 *c, void *ws, size_t ws_bytes, void *stream,
+                             const cqt::SliceSource *src = nullptr) {
     Call k;
     cqt_status s = begin_call(p, x, x_stride, batch, valid_len, c, ws, ws_bytes, stream, k);
     if (s != CQT_OK) return s;
-    cudaError_t e = launch_rfft_forward(*p, x, x_stride, batch, valid_len, k.T, k.second, k.st);
+    cudaError_t e = launch_rfft_forward(*p, x, x_stride, batch, valid_len, k.T, k.second, k.st, src);
     if (e == cudaSuccess) e = launch_bands_from_spectrum(*p, table, k.second, reinterpret_cast<float2 *>(c), k.huge, batch, k.st);
     return end_call(k, e);
 }
@@ -685,6 +686,18 @@ cqt_status run_synthesis_form(const cqt_plan *p, const float *table, bool fold, 
 }
 
 }  // namespace
+
+namespace cqt {
+
+// Analysis of slices cut from a stream's ring buffer (slicq.cu): cqt_analyse with the slice cut fused into the load of
+// the long FFT's first pass.  batch = slices x channels rows of the plan's full length.
+cqt_status analyse_slices(const cqt_plan *p, const SliceSource &src, int64_t batch, cqt_c64 *c, void *ws, size_t ws_bytes,
+                          void *stream) {
+    if (!p || !src.ring || !src.win || !can_fuse_slice_cut(*p)) return CQT_ERR_INVALID_ARG;
+    return run_analysis_form(p, p->d.tab_analysis, src.ring, p->N, batch, p->N, c, ws, ws_bytes, stream, &src);
+}
+
+}  // namespace cqt
 
 extern "C" {
 

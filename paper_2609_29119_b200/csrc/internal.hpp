@@ -103,8 +103,19 @@ enum { TAB_ANALYSIS = 0, TAB_SYNTHESIS = 1, TAB_ANALYSIS_ADJ = 2, TAB_SYNTHESIS_
 void note_launch(const cqt_plan &p, const char *name, cudaStream_t st);
 
 // long_fft.cu
+// Input of the forward long FFT taken from a ring buffer of a stream instead of signal rows (sliced transform, slice
+// cut fused into the load): row r = slice r / channels of channel r % channels; sample i of that slice is
+// win[i] * ring[channel * ring_len + (first + (r / channels) * hop + i) mod ring_len], zero before the stream's start.
+struct SliceSource {
+    const float *ring;
+    const float *win;
+    long long ring_len, first, hop;
+    int channels;
+};
+// src != nullptr needs a plan whose long FFT runs in two passes (can_fuse_slice_cut)
 cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,
-                                float2 *T, float2 *X, cudaStream_t st);
+                                float2 *T, float2 *X, cudaStream_t st, const SliceSource *src = nullptr);
+inline bool can_fuse_slice_cut(const cqt_plan &p) { return p.lf.A > 1; }
 cudaError_t launch_rfft_inverse(const cqt_plan &p, const float2 *Y, float2 *T, float *x, int64_t x_stride,
                                 int64_t batch, int64_t valid_len, cudaStream_t st);
 // The dynamic shared-memory limit is a property of the kernel function, shared by every plan of the process: it is

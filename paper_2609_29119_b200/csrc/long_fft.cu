@@ -58,6 +58,13 @@ struct LongArgs {
     float scale;
     uint32_t cols_magic, rows_magic;
     int *dbg;
+    // sliced source (forward column pass of the streaming form): row r is slice r / channels of channel r % channels,
+    // its sample i is slice_win[i] * ring[channel][(slice_first + (r / channels) * hop + i) mod ring_len], zero
+    // before the start of the stream
+    const float *ring;
+    const float *slice_win;
+    long long ring_len, slice_first, hop;
+    int channels;
 };
 
 __device__ __forceinline__ float2 load_packed(const float *row, int j, int valid_len, int aligned) {
@@ -106,26 +113,52 @@ using Sh_16_8_8_8_9 = Shape<16, 8, 8, 8, 9>;
 
 // The host picks the instantiation that matches the plan (pick_kernel below): a kernel holds the code of one shape only.
 // ---------------------------------------------------------------- forward, pass C
-template <class SH>
+// SLICED: the rows are slices cut from a ring buffer of the stream and multiplied by the slice window on load
+// (the slice cut of the sliced transform, fused into this pass: no staged copy of the windowed slices)
+template <class SH, bool SLICED>
 __device__ __forceinline__ void cols_fwd_body(const LongArgs &a, const FftPlan &fp, float2 *buf, const float2 *tws,
                                               const float2 *wl, int j2_0, int ch, int tid, int nthr) {
     const int TW = a.tw_cols;
-    const float *row = a.x_in + (long long)ch * a.x_stride;
     float2 *T = a.T + (long long)ch * a.t_pitch;
-    auto load = [&](int j1, int c) -> float2 { return load_packed(row, j1 * a.B + j2_0 + c, a.valid_len, a.aligned); };
     auto store = [&](int k1, int c, float2 v) {
         const float2 w = twiddle_s(wl, a.log_lp_c, (uint32_t)(j2_0 + c) * (uint32_t)k1);
         if (CQT_CHK(a.dbg, 201, k1 * a.B + j2_0 + c, a.Lp)) T[k1 * a.B + j2_0 + c] = cmul(v, w);
     };
-    if constexpr (SH::is_static) {
-        tile_fft_static<SH, -1, true, false>(buf, tws, load, store, tid, nthr);
+    auto run = [&](auto load) {
+        if constexpr (SH::is_static) {
+            tile_fft_static<SH, -1, true, false>(buf, tws, load, store, tid, nthr);
+        } else {
+            const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
+            fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+        }
+    };
+    if constexpr (SLICED) {
+        const int s_rel = ch / a.channels, chan = ch - s_rel * a.channels;
+        const long long first = a.slice_first + (long long)s_rel * a.hop;   // stream index of the slice's sample 0
+        const float *ring = a.ring + (long long)chan * a.ring_len;
+        // position of sample 0 in the ring; the slice is no longer than the ring, so one conditional subtraction wraps
+        const int R = (int)a.ring_len;
+        const int base = (int)(((first % a.ring_len) + a.ring_len) % a.ring_len);
+        const int lead = first < 0 ? (int)(-first) : 0;                      // samples before the start of the stream
+        const float *win = a.slice_win;
+        auto sample = [&](int i) -> float {
+            if (i < lead) return 0.f;
+            int p = base + i;
+            if (p >= R) p -= R;
+            if (!CQT_CHK(a.dbg, 212, p, R)) return 0.f;
+            return __ldg(win + i) * __ldg(ring + p);
+        };
+        run([&](int j1, int c) -> float2 {
+            const int i = 2 * (j1 * a.B + j2_0 + c);
+            return make_float2(sample(i), sample(i + 1));
+        });
     } else {
-        const Tile t{buf, TW, TW, a.cols_magic, a.A * TW, a.dbg};
-        fft_fused<-1, BlockSync, true, false, true, false, true, true>(t, fp, tws, load, store, tid, nthr);
+        const float *row = a.x_in + (long long)ch * a.x_stride;
+        run([&](int j1, int c) -> float2 { return load_packed(row, j1 * a.B + j2_0 + c, a.valid_len, a.aligned); });
     }
 }
 
-template <class SH>
+template <class SH, bool SLICED = false>
 __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
@@ -139,7 +172,7 @@ __global__ void __launch_bounds__(512, 2) rfft_cols_fwd_kernel(LongArgs a) {
     stage_full(tws, a.tw, fp, tid, nthr);
     stage_table(wl, a.tw + a.tw_lp, a.n_lp, tid, nthr);
     pdl_wait();   // the tables above belong to the plan; what follows reads the predecessor's output
-    cols_fwd_body<SH>(a, fp, buf, tws, wl, j2_0, ch, tid, nthr);
+    cols_fwd_body<SH, SLICED>(a, fp, buf, tws, wl, j2_0, ch, tid, nthr);
 }
 
 // Rows of CTA t of the forward row kernel, column r of its tile: r < TW is row TW t + 1 + r, r >= TW its mirror
@@ -522,7 +555,8 @@ struct PickKernel<K, SH, Rest...> {
         return SH::matches(fp, ncols) ? (const void *)K<SH>::fn : PickKernel<K, Rest...>::get(fp, ncols);
     }
 };
-template <class SH> struct ColsFwdK { static constexpr auto fn = rfft_cols_fwd_kernel<SH>; };
+template <class SH> struct ColsFwdK { static constexpr auto fn = rfft_cols_fwd_kernel<SH, false>; };
+template <class SH> struct ColsFwdSlicedK { static constexpr auto fn = rfft_cols_fwd_kernel<SH, true>; };
 template <class SH> struct RowsFwdK { static constexpr auto fn = rfft_rows_fwd_kernel<SH>; };
 template <class SH> struct RowsInvK { static constexpr auto fn = irfft_rows_kernel<SH>; };
 template <class SH> struct ColsInvK { static constexpr auto fn = irfft_cols_kernel<SH>; };
@@ -530,6 +564,10 @@ template <class SH> struct ColsInvK { static constexpr auto fn = irfft_cols_kern
 static const void *cols_fwd_fn(const cqt_plan &p) {
     return PickKernel<ColsFwdK, Sh_8_8_8_16_16, Sh_16_16_1_16_16, Sh_16_8_1_16_16, Sh_16_8_8_8_8, Sh_16_16_8_8_8>::get(
         p.ffts[p.lf.fft_A], p.lf.tw_cols);
+}
+// the slice lengths in use give 16 x 8 or 16 x 16 or 8 x 8 x 8 tiles; other plans take the run-time planned instantiation
+static const void *cols_fwd_sliced_fn(const cqt_plan &p) {
+    return PickKernel<ColsFwdSlicedK, Sh_8_8_8_16_16, Sh_16_16_1_16_16, Sh_16_8_1_16_16>::get(p.ffts[p.lf.fft_A], p.lf.tw_cols);
 }
 static const void *rows_fwd_fn(const cqt_plan &p) {
     const int ncols = p.lf.A == 1 ? 1 : 2 * p.lf.tw_rows;
@@ -559,15 +597,20 @@ static int threads_for(size_t elements, const FftPlan &fp) {
 }
 
 cudaError_t launch_rfft_forward(const cqt_plan &p, const float *x, int64_t x_stride, int64_t batch, int64_t valid_len,
-                                float2 *T, float2 *X, cudaStream_t st) {
+                                float2 *T, float2 *X, cudaStream_t st, const SliceSource *src) {
     LongArgs a = base_args(p, valid_len, x_stride, x);
     a.x_in = x;
     a.T = T;
     a.X = X;
     const LongFft &lf = p.lf;
+    if (src) {
+        if (lf.A == 1 || src->channels <= 0 || src->ring_len < p.N) return cudaErrorInvalidValue;
+        a.ring = src->ring; a.slice_win = src->win;
+        a.ring_len = src->ring_len; a.slice_first = src->first; a.hop = src->hop; a.channels = src->channels;
+    }
     if (lf.A > 1) {
         dim3 grid((unsigned)(lf.B / lf.tw_cols), (unsigned)batch);
-        launch_long(cols_fwd_fn(p), grid, threads_for((size_t)lf.A * lf.tw_cols, p.ffts[lf.fft_A]), cols_smem(p), a, st);
+        launch_long(src ? cols_fwd_sliced_fn(p) : cols_fwd_fn(p), grid, threads_for((size_t)lf.A * lf.tw_cols, p.ffts[lf.fft_A]), cols_smem(p), a, st);
         note_launch(p, "rfft_cols_fwd", st);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -621,6 +664,8 @@ cudaError_t configure_long_fft_kernels(const cqt_plan &p) {
     if (e != cudaSuccess) return e;
     if (p.lf.A > 1) {
         e = allow_dynamic_smem(cols_fwd_fn(p), cols_smem(p), p);
+        if (e != cudaSuccess) return e;
+        e = allow_dynamic_smem(cols_fwd_sliced_fn(p), cols_smem(p), p);
         if (e != cudaSuccess) return e;
         e = allow_dynamic_smem(cols_inv_fn(p), cols_smem(p), p);
     }

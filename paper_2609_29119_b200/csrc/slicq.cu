@@ -12,6 +12,12 @@
 #include "engine.cuh"
 #include "internal.hpp"
 
+namespace cqt {
+// api.cu: cqt_analyse on slices cut from a ring buffer, the cut fused into the load of the long FFT's first pass
+cqt_status analyse_slices(const cqt_plan *p, const SliceSource &src, int64_t batch, cqt_c64 *c, void *ws, size_t ws_bytes,
+                          void *stream);
+}  // namespace cqt
+
 struct cqt_slicq {
     const cqt_plan *plan = nullptr;
     int C = 0;
@@ -136,12 +142,20 @@ cqt_status analyse_ready(cqt_slicq *s, cudaStream_t st) {
         // slices whose coefficient slots are consecutive in memory
         const int64_t slot = s->next_slice % s->K;
         const int64_t cnt = std::min<int64_t>(ready - s->next_slice, s->K - slot);
-        dim3 grid(blocks_for(s->sl), (unsigned)(cnt * s->C));
-        if (cqt::launch_kernel_args(slicq_cut_kernel, grid, dim3(256), 0, st, s->d_in, s->ring_in, s->d_win, s->d_stage, s->sl, s->H,
-                               s->next_slice, s->C) != cudaSuccess)
-            return CQT_ERR_CUDA;
-        cqt_status r = cqt_analyse(s->plan, s->d_stage, s->sl, cnt * s->C, s->sl,
-                                   s->d_coef + slot * s->C * cqt_plan_coeff_count(s->plan), s->d_ws, s->ws_bytes, st);
+        cqt_c64 *coef = s->d_coef + slot * s->C * cqt_plan_coeff_count(s->plan);
+        cqt_status r;
+        if (cqt::can_fuse_slice_cut(*s->plan) && s->ring_in >= s->sl) {
+            // the slice cut (window x ring samples) happens in the load of the long FFT's first pass
+            const cqt::SliceSource src{s->d_in, s->d_win, s->ring_in, s->next_slice * s->H - s->H, s->H, s->C};
+            r = cqt::analyse_slices(s->plan, src, cnt * s->C, coef, s->d_ws, s->ws_bytes, st);
+        } else {
+            // short slices (one-pass long FFT): a kernel of its own writes the windowed slices to a staging buffer
+            dim3 grid(blocks_for(s->sl), (unsigned)(cnt * s->C));
+            if (cqt::launch_kernel_args(slicq_cut_kernel, grid, dim3(256), 0, st, s->d_in, s->ring_in, s->d_win, s->d_stage, s->sl,
+                                        s->H, s->next_slice, s->C) != cudaSuccess)
+                return CQT_ERR_CUDA;
+            r = cqt_analyse(s->plan, s->d_stage, s->sl, cnt * s->C, s->sl, coef, s->d_ws, s->ws_bytes, st);
+        }
         if (r != CQT_OK) return r;
         s->next_slice += cnt;
     }

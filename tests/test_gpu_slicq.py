@@ -12,14 +12,19 @@ pytestmark = pytest.mark.gpu
 W = small_workload("slices_4096", N=4096, valid_len=4096, fs=22050.0, fmin=100.0, fmax=11025.0, bins_per_octave=12,
                    m_policy=wl.M_SMOOTH, channels=2, kind="pink_notes", slice_len=4096, transition=512,
                    stream_len=5 * 4096 + 123)
+# a slice long enough for the two-pass long FFT, where the slice cut is fused into the first pass's load
+W16 = small_workload("slices_16384", N=16384, valid_len=16384, fs=44100.0, fmin=60.0, fmax=22050.0, bins_per_octave=12,
+                     m_policy=wl.M_SMOOTH, channels=2, kind="pink_notes", slice_len=16384, transition=4096,
+                     stream_len=4 * 16384 + 321)
+BOTH = pytest.mark.parametrize("w", [W, W16], ids=lambda w: w.name)
 
 
-def _stream(plan, x, chunks, K=4, pull_every=1):
+def _stream(plan, x, chunks, K=4, pull_every=1, w=W):
     from paper_2609_29119_b200 import SliCQ
-    sq = SliCQ(plan, x.shape[0], W.transition, K)
+    sq = SliCQ(plan, x.shape[0], w.transition, K)
     xd = torch.from_numpy(x).cuda()
     n = x.shape[1]
-    out = torch.zeros((x.shape[0], n + 2 * W.slice_len), device="cuda")
+    out = torch.zeros((x.shape[0], n + 2 * w.slice_len), device="cuda")
     got, pos, i = 0, 0, 0
     coeffs = {}
     while pos < n:
@@ -40,16 +45,17 @@ def _stream(plan, x, chunks, K=4, pull_every=1):
     return out[:, :got].cpu().numpy(), coeffs, nbytes
 
 
-def test_streaming_matches_offline_slicing():
-    lay = oracle_layout(W)
-    plan = library_plan(W)
-    x = wl.make_signal(W)
+@BOTH
+def test_streaming_matches_offline_slicing(w):
+    lay = oracle_layout(w)
+    plan = library_plan(w)
+    x = wl.make_signal(w)
     n = x.shape[1]
-    H = W.slice_len // 2
-    y, coeffs, _ = _stream(plan, x, [H])
+    H = w.slice_len // 2
+    y, coeffs, _ = _stream(plan, x, [H], w=w)
     assert y.shape[1] >= n
     # oracle: cut, per-slice T and S, overlap-add
-    slices = orc.slicq_cut(x.astype(np.float64), W.slice_len, W.transition)       # [C, ns, sl]
+    slices = orc.slicq_cut(x.astype(np.float64), w.slice_len, w.transition)       # [C, ns, sl]
     for s, c in coeffs.items():
         want = orc.analyse(lay, slices[:, s, :])
         errs = band_rel_errors(lay, c, want)
@@ -62,18 +68,19 @@ def test_streaming_matches_offline_slicing():
     plan.close()
 
 
-def test_chunking_does_not_change_the_result_and_memory_is_bounded():
-    plan = library_plan(W)
-    x = wl.make_signal(W)
-    H = W.slice_len // 2
-    y1, _, b1 = _stream(plan, x, [H])
-    y2, _, b2 = _stream(plan, x, [1, 7, H - 3, 3 * H + 5, 200], pull_every=2)
+@BOTH
+def test_chunking_does_not_change_the_result_and_memory_is_bounded(w):
+    plan = library_plan(w)
+    x = wl.make_signal(w)
+    H = w.slice_len // 2
+    y1, _, b1 = _stream(plan, x, [H], w=w)
+    y2, _, b2 = _stream(plan, x, [1, 7, H - 3, 3 * H + 5, 200], pull_every=2, w=w)
     m = min(y1.shape[1], y2.shape[1])
     assert m >= x.shape[1]
     assert np.array_equal(y1[:, :m], y2[:, :m])
     # a stream three times as long uses the same device memory
-    x3 = wl.make_signal(W, length=3 * x.shape[1])
-    y3, _, b3 = _stream(plan, x3, [2 * H])
+    x3 = wl.make_signal(w, length=3 * x.shape[1])
+    y3, _, b3 = _stream(plan, x3, [2 * H], w=w)
     assert b1 == b2 == b3
     assert snr_db(x3, y3[:, :x3.shape[1]]).min() >= 120.0
     plan.close()
